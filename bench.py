@@ -1,0 +1,331 @@
+#!/usr/bin/env python
+"""Benchmark of the Local AdaAlter hot path (Algorithm 3 of arXiv 1911.09030) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+
+A "step" is one `la_run(T)` of the chosen configuration: T iterations of Algorithm 3 for all
+W workers over all N coordinates, including the synchronisations that fall in it.  Prints ONE
+JSON line.  With N > 1 GPUs (torchrun) each rank runs the same configuration on its own
+coordinate range (coordinates never interact, so there is no data-path collective): weak
+scaling.  `--impl reference` times the CPU oracle, as it stands, on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "worker_param_updates_per_sec"
+UNIT = "worker*param updates/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs (read-only)."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: str):
+        self.idx = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.idx)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._pump, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        rows = [l for (ts, l) in self.lines if t0 <= ts <= t1 + 0.2] or [l for _, l in self.lines]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in rows:
+            f = [v.strip() for v in l.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- oracle leg
+def oracle_rate(wl, n_slice: int, threads: int = 1, T=None):
+    """worker*param updates/s of the CPU oracle on the first n_slice coordinates at full W and T."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle.oracle import Oracle
+    T = wl.T if T is None else T
+    per = n_slice // threads
+    jobs = []
+    for k in range(threads):
+        lo = k * per
+        arr = wl.arrays(lo, per)
+        o = Oracle(per, wl.W, wl.eta, wl.eps, wl.H, wl.b0sq, j_base=lo)
+        if wl.grad == "quadratic":
+            o.set_grad_quadratic(wl.noise_seed, arr["a"], arr["c"], wl.sigma)
+        elif wl.grad == "noise_scaled":
+            o.set_grad_noise(wl.noise_seed, arr["s"])
+        else:
+            o.set_grad_noise(wl.noise_seed, None)
+        if wl.bf16_grads:
+            o.set_grad_bf16(True)
+        jobs.append(o)
+    t0 = time.perf_counter()
+    if threads == 1:
+        jobs[0].run(T)
+    else:
+        with ThreadPoolExecutor(threads) as ex:
+            list(ex.map(lambda o: o.run(T), jobs))
+    dt = time.perf_counter() - t0
+    return per * threads * wl.W * T / dt, dt
+
+
+def run_reference(args, wl):
+    """The reference arm: the oracle (plain single-threaded C++), timed as it stands."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_slice = min(wl.N, 1 << 14)
+    for _ in range(args.warmup):
+        oracle_rate(wl, 1024)
+    rates, t_all = [], 0.0
+    for _ in range(args.steps):
+        r, dt = oracle_rate(wl, n_slice)
+        rates.append(r); t_all += dt
+    value = float(np.mean(rates))
+    sample = f"first {n_slice} coordinates of {wl.name} at full W={wl.W}, T={wl.T}, per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_all / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_config(wl, args),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(wl, args):
+    return {"workload": f"{wl.name}: W={wl.W}, N={wl.N} fp32 in {len(wl.sizes)} tensor(s), grad={wl.grad}"
+                        f"{'+bf16' if wl.bf16_grads else ''}, eta={wl.eta}, eps={wl.eps}, H={wl.H}, T={wl.T} per step",
+            "W": wl.W, "N": wl.N, "H": wl.H, "T": wl.T, "fusion": getattr(args, "fusion", None),
+            "l2": "inputs larger than L2 (state %.2f GiB per GPU)" % (wl.N * 4 * (2 * wl.W + 1) / 2 ** 30),
+            "sharding": "by coordinate range, no collective"}
+
+
+# --------------------------------------------------------------------------- CUDA leg
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_1911_09030_b200 import local_adaalter as la
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # this rank's coordinate range: the same configuration, shifted (weak scaling)
+    j_base = rank * ((wl.N + 3) // 4 * 4)
+    arr = wl.arrays()            # same per-coordinate inputs on every rank; noise differs through j_base
+    stream = torch.cuda.current_stream()
+    ctx = la.LocalAdaAlter.with_torch_arena(wl.sizes, wl.W, wl.eta, wl.eps, wl.H, b0sq=wl.b0sq, j_base=j_base)
+
+    pinned = {k: torch.from_numpy(v).pin_memory() for k, v in arr.items()}
+    x0_pin = torch.zeros(wl.N, dtype=torch.float32).pin_memory()
+    out_pin = {k: torch.empty(wl.N, dtype=torch.float32).pin_memory() for k in ("x", "b2", "bs")}
+
+    def upload():
+        ctx._ck(ctx.L.la_set_init(ctx.h, x0_pin.data_ptr(), float(wl.b0sq)))
+        if wl.grad == "quadratic":
+            ctx._ck(ctx.L.la_set_grad_quadratic(ctx.h, wl.noise_seed, pinned["a"].data_ptr(),
+                                                 pinned["c"].data_ptr(), float(wl.sigma)))
+        elif wl.grad == "noise_scaled":
+            ctx._ck(ctx.L.la_set_grad_noise(ctx.h, wl.noise_seed, pinned["s"].data_ptr()))
+        else:
+            ctx._ck(ctx.L.la_set_grad_noise(ctx.h, wl.noise_seed, None))
+    h2d = 4 * wl.N * (1 + len(arr))
+    d2h = 4 * wl.N * 3
+
+    upload()
+    if wl.bf16_grads:
+        ctx.set_grad_dtype(la.LA_BF16)
+    ctx.set_fusion(args.fusion)
+    if args.blocks_per_sm:
+        ctx.set_launch_shape(args.blocks_per_sm)
+
+    # ---- device-resident timing -----------------------------------------------------------
+    for _ in range(args.warmup):
+        ctx.run(wl.T)
+    barrier()
+    ctx.get_stats(reset=True)
+    ctx.set_profiling(True)
+    vis = [v for v in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if v]
+    sampler = ClockSampler(vis[local_rank] if local_rank < len(vis) else str(local_rank))
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.time()
+    e0.record(stream)
+    for _ in range(args.steps):
+        ctx.run(wl.T)
+    e1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    ms_total = e0.elapsed_time(e1)
+    stats = ctx.get_stats(reset=True)
+    ctx.set_profiling(False)
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+
+    # ---- end to end through the C-ABI with host buffers -------------------------------------
+    def e2e_step():
+        upload()
+        ctx.run(wl.T)
+        ctx._ck(ctx.L.la_read_state(ctx.h, 0, out_pin["x"].data_ptr(), out_pin["b2"].data_ptr(),
+                                    out_pin["bs"].data_ptr()))
+    e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    e2e_steps = max(1, min(args.steps, 3))
+    for _ in range(e2e_steps):
+        e2e_step()                               # la_read_state synchronises the stream
+    barrier()
+    e2e_ms = 1e3 * (time.perf_counter() - t0) / e2e_steps
+
+    t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = float(t[0]), float(t[1])
+    ms_per_step = ms_total / args.steps
+    units = wl.W * wl.N * wl.T * world
+    value = units / (ms_per_step * 1e-3)
+
+    if rank == 0:
+        peak, peak_kind = measured_peak()
+        launches = {k: stats[k] for k in ("launches_local", "launches_sync", "launches_fused")}
+        n_local = max(1, stats["launches_local"])
+        ms_local = stats["ms_local"] / n_local
+        bytes_local = stats["bytes_local"] / n_local
+        achieved = bytes_local / (ms_local * 1e-3) / 1e9 if ms_local > 0 else None
+        roofline = {
+            "bound": "hbm", "kernel": "la_sweep<STEP> (K1 local step)", "achieved": achieved, "peak": peak,
+            "peak_kind": peak_kind, "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
+            "traffic": None, "bytes_per_launch": bytes_local, "ms_per_launch": ms_local,
+            "bytes_per_update": bytes_local / (wl.W * wl.N),
+        }
+        per_class = {}
+        for cls in ("local", "sync", "fused"):
+            n = stats[f"launches_{cls}"]
+            if n:
+                ms = stats[f"ms_{cls}"] / n
+                per_class[cls] = {"launches": n, "ms_per_launch": ms,
+                                  "GBps": stats[f"bytes_{cls}"] / n / (ms * 1e-3) / 1e9 if ms > 0 else None,
+                                  "share_of_device_time": None}
+        tot = sum(stats[f"ms_{c}"] for c in ("local", "sync", "fused"))
+        for cls in per_class:
+            per_class[cls]["share_of_device_time"] = stats[f"ms_{cls}"] / tot if tot > 0 else None
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            n_slice = min(wl.N, 1 << 16)
+            v, dt = oracle_rate(wl, n_slice)
+            cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt,
+                   "sample": f"first {n_slice} coordinates of {wl.name} at full W={wl.W}, T={wl.T}"}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(wl, args),
+            "clocks": clocks,
+            "e2e": {"value": units / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+            "gpu_launches": int(sum(launches.values())),
+            "roofline": roofline, "cpu_baseline": cpu, "kernels": per_class,
+            "hbm_GBps_whole_step": (stats["bytes_local"] + stats["bytes_sync"] + stats["bytes_fused"]) / (ms_total * 1e-3) / 1e9,
+        }
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--H", type=int, default=None, help="override the synchronisation period")
+    ap.add_argument("--T", type=int, default=None, help="override iterations per step")
+    ap.add_argument("--fusion", type=int, default=1, help="0 unfused, 1 step+sync, 2 sync+next step")
+    ap.add_argument("--blocks-per-sm", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_1911_09030_b200 import workloads
+    wl = workloads.config(args.workload)
+    if args.H is not None:
+        wl.H = args.H
+    if args.T is not None:
+        wl.T = args.T
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

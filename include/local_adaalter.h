@@ -1,0 +1,162 @@
+/*
+ * local_adaalter.h — C-ABI of the Local AdaAlter hot-path library (CUDA, sm_100a).
+ *
+ * The library simulates W data-parallel workers on ONE GPU: every worker owns a
+ * replica of a flat fp32 parameter vector x (N coordinates, the concatenation of
+ * K tensors) and of the squared-gradient accumulator B^2; one further array holds
+ * the accumulator as of the last synchronisation, which Algorithm 3 of
+ * arXiv 1911.09030 uses as the (worker-independent) denominator.  All state lives
+ * in device memory and every arithmetic step of the method runs in CUDA kernels.
+ *
+ * Conventions
+ *   - Every function returns an int status: LA_OK (0) or a negative LA_E* code.
+ *     Nothing throws, aborts or traps.  la_last_error() gives the message of the
+ *     most recent failure on a context (or of the last failed la_create*).
+ *   - "host" pointers are ordinary CPU memory (pinned or pageable); "device"
+ *     pointers are CUDA global memory of the context's device.  Unless stated
+ *     otherwise the library copies what it is given and keeps no reference.
+ *   - A context is bound to one device and one stream; all kernels are enqueued
+ *     on that stream.  One caller thread at a time per context.
+ *   - Calls that only enqueue work return before it finishes (la_local_step,
+ *     la_sync, la_run, the la_set_* uploads); la_read_state, la_get_stats and
+ *     la_destroy synchronise the stream.
+ *   - Rounding contract (what "the same result" means): fp32 IEEE-754, one
+ *     rounding per written operation, fused multiply-add where stated:
+ *       eps2 = eps*eps;  q = (float)t' * eps2;  d = B2stale[j] + q;
+ *       r = eta_t / sqrtf(d);  x = fmaf(-r, g, x);  B2 = fmaf(g, g, B2);
+ *       mean over workers = adjacent-pair tree sum, then one division by (float)W.
+ */
+#ifndef LOCAL_ADAALTER_H_
+#define LOCAL_ADAALTER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct la_ctx la_ctx; /* opaque; owned by the library until la_destroy */
+
+enum {
+  LA_OK = 0,
+  LA_EINVAL = -1, /* bad argument (NULL handle, N=0, W=0, H=0, eps<=0, non-finite eta, ...) */
+  LA_ENOMEM = -2, /* device or host allocation failed, or caller arena too small */
+  LA_ECUDA = -3,  /* a CUDA runtime call failed; message in la_last_error */
+  LA_ESTATE = -4  /* call not valid in the context's current configuration */
+};
+
+enum { LA_F32 = 0, LA_BF16 = 1 };               /* gradient dtype */
+enum { LA_FUSE_NONE = 0, LA_FUSE_STEP_SYNC = 1, /* la_run: step t'=H and its sync in one pass */
+       LA_FUSE_SYNC_STEP = 2 };                 /* la_run: sync folded into the following step */
+#define LA_H_NEVER 0xFFFFFFFFu                  /* H = +infinity: never synchronise */
+#define LA_MAX_WORKERS 64u
+
+/* Extended creation parameters.  Zero-initialise, then fill. */
+typedef struct la_config {
+  uint32_t K;            /* number of tensors (>= 1) */
+  const uint64_t* sizes; /* host, K entries, each >= 1; tensors are packed back to back, N = sum */
+  uint64_t j_base;       /* global index of coordinate 0 (multiple of 4); the noise of coordinate j
+                            is keyed on j_base + j, so a job can be sharded by coordinate range */
+  uint32_t W;            /* workers / replicas, 1..LA_MAX_WORKERS */
+  uint32_t H;            /* synchronisation period (Algorithm 3), >= 1; LA_H_NEVER = never */
+  float eta;             /* learning rate (finite) */
+  float eps;             /* epsilon (> 0); the algorithm uses eps^2 */
+  float b0sq;            /* b_0^2 >= 0, initial value of every accumulator (Algorithm 3, init) */
+  void* dev_arena;       /* device; optional caller-owned state memory (256-byte aligned), or NULL */
+  uint64_t arena_bytes;  /* size of dev_arena; must be >= la_arena_bytes() */
+  void* stream;          /* a cudaStream_t, or NULL for the legacy default stream */
+  int32_t device;        /* CUDA device ordinal, or -1 for the current device */
+} la_config;
+
+typedef struct la_stats {
+  uint64_t launches_local;  /* K1: local step (gradient + update + accumulate), Algorithm 3 body */
+  uint64_t launches_sync;   /* K2: stand-alone synchronisation */
+  uint64_t launches_fused;  /* K3/K4: a local step and a synchronisation in one pass */
+  uint64_t launches_other;  /* fills, scatter/gather of state */
+  double ms_local, ms_sync, ms_fused; /* device time per class; only while profiling is on */
+  double bytes_local, bytes_sync, bytes_fused; /* algorithmic HBM bytes issued per class */
+} la_stats;
+
+/* ---- creation / destruction ------------------------------------------------
+ * Algorithm 3, initialisation line: x_{i,0} = x_0, B^2_{i,0} = b_0^2 * 1.
+ * la_create: one tensor of N coordinates, x_0 = 0, b_0^2 = 0, device memory
+ * allocated (and later freed) by the library, current device, default stream. */
+int la_create(la_ctx** out, uint64_t N, uint32_t W, float eta, float eps, uint32_t H);
+int la_create_ex(la_ctx** out, const la_config* cfg);
+/* Bytes of device memory a context with this configuration needs (state only). */
+int la_arena_bytes(const la_config* cfg, uint64_t* bytes);
+/* Frees library-owned memory only; a caller arena is left untouched.  NULL is allowed. */
+void la_destroy(la_ctx* ctx);
+/* Message of the last error; ctx may be NULL (then: last failed creation in this thread). */
+const char* la_last_error(const la_ctx* ctx);
+
+/* ---- configuration ---------------------------------------------------------
+ * Re-initialise the state: every replica gets x0 (host, N floats; NULL = zeros), every
+ * accumulator and the stale accumulator get b0sq; counters return to zero. */
+int la_set_init(la_ctx* ctx, const float* x0_host, float b0sq);
+/* Synthetic stochastic gradient (stands in for G_{i,t} = grad f(x_{i,t-1}; z_{i,t}) of
+ * Algorithm 3): g = s_j * xi, xi ~ N(0,1) from a counter-based generator keyed on
+ * (seed, worker, step, global coordinate).  s_host: N floats or NULL for s == 1. */
+int la_set_grad_noise(la_ctx* ctx, uint64_t seed, const float* s_host);
+/* Noisy diagonal quadratic f = 1/2 sum a_j (x_j - c_j)^2: g = a_j (x - c_j) + sigma * xi,
+ * evaluated at the worker's own iterate.  a_host, c_host: N floats each. */
+int la_set_grad_quadratic(la_ctx* ctx, uint64_t seed, const float* a_host, const float* c_host,
+                          float sigma);
+/* Deterministic gradient g = s_j on every worker and step (s_host NULL = 1); for closed-form tests. */
+int la_set_grad_constant(la_ctx* ctx, const float* s_host);
+/* LA_BF16: round every generated gradient to bfloat16 (nearest-even) and widen, in registers. */
+int la_set_grad_dtype(la_ctx* ctx, int dtype);
+/* Test switch: all workers draw worker 0's noise (then replicas stay bitwise equal). */
+int la_set_identical_workers(la_ctx* ctx, int on);
+/* Warm-up of Section 6.2: eta_t = eta * min(1, t / warm_up_steps); 0 switches it off. */
+int la_set_warmup(la_ctx* ctx, uint32_t warm_up_steps);
+/* How la_run realises the synchronisation (LA_FUSE_*); results are bitwise the same. */
+int la_set_fusion(la_ctx* ctx, int mode);
+/* Tuning knob: the sweep kernels run as a grid-stride loop over at most
+ * blocks_per_sm * (number of SMs) blocks of 256 threads (default 8). */
+int la_set_launch_shape(la_ctx* ctx, int blocks_per_sm);
+/* Record CUDA events around every launch and accumulate device time per class. */
+int la_set_profiling(la_ctx* ctx, int on);
+
+/* ---- the hot path ------------------------------------------------------------
+ * One iteration of Algorithm 3 WITHOUT its synchronisation branch, for every worker:
+ * t += 1, t' += 1; G at the worker's own x; y = x - eta_t G / sqrt(B2stale + t' eps^2);
+ * A^2 = B^2 + G o G; both committed locally. */
+int la_local_step(la_ctx* ctx);
+/* Same, with G_{i,t} supplied by the caller: device pointer to [W][N] gradients, worker-major,
+ * dtype LA_F32 (4 bytes) or LA_BF16 (2 bytes, widened exactly).  16-byte aligned. Not retained
+ * beyond the kernel; the caller must keep it alive until the stream reaches that point. */
+int la_local_step_grads(la_ctx* ctx, const void* g_dev, int dtype);
+/* Synchronisation branch of Algorithm 3: x and B^2 of every worker are replaced by the means
+ * over workers; the mean B^2 becomes the stale denominator; t' = 0; n_sync += 1.  Legal at any
+ * time (outside la_run it need not fall on a multiple of H). */
+int la_sync(la_ctx* ctx);
+/* T iterations of Algorithm 3: repeat { local step; if t' == H: synchronise }.  May use fused
+ * kernels; the state afterwards is bitwise that of the unfused sequence. */
+int la_run(la_ctx* ctx, uint64_t T);
+
+/* ---- state access (synchronises the stream) ------------------------------------
+ * Copy worker `worker`'s x and B^2 and the shared stale accumulator to host buffers of N floats
+ * each, in packed tensor order.  Any pointer may be NULL. */
+int la_read_state(la_ctx* ctx, uint32_t worker, float* x_host, float* b2_host, float* bs_host);
+/* The reverse (checkpoint restore).  Any pointer may be NULL. */
+int la_write_state(la_ctx* ctx, uint32_t worker, const float* x_host, const float* b2_host,
+                   const float* bs_host);
+/* Read coordinates [j0, j0+n) only. */
+int la_read_range(la_ctx* ctx, uint32_t worker, uint64_t j0, uint64_t n, float* x_host,
+                  float* b2_host, float* bs_host);
+/* Offset (in coordinates) and size of tensor k inside the packed vector. */
+int la_tensor_range(const la_ctx* ctx, uint32_t k, uint64_t* offset, uint64_t* size);
+/* t = local steps since creation, t_prime = local steps since the last synchronisation,
+ * n_sync = synchronisations so far.  (Algorithm 3's t' of the NEXT step is t_prime + 1.) */
+int la_get_counters(const la_ctx* ctx, uint64_t* t, uint32_t* t_prime, uint64_t* n_sync);
+int la_set_counters(la_ctx* ctx, uint64_t t, uint32_t t_prime, uint64_t n_sync);
+/* Launch counts, algorithmic bytes and (when profiling) device milliseconds per kernel class.
+ * reset != 0 clears the counters after reading. */
+int la_get_stats(la_ctx* ctx, la_stats* out, int reset);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOCAL_ADAALTER_H_ */

@@ -1,0 +1,581 @@
+// C-ABI of the Local AdaAlter hot-path library: context, schedule (Algorithm 3's outer
+// loop and its t / t' / sync bookkeeping), state upload/download and kernel dispatch.
+// All arithmetic of the method lives in la_sweep.cuh; this file moves scalars and pointers.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/local_adaalter.h"
+#include "la_sweep.cuh"
+
+namespace la {
+
+SweepFn lookup_sweep_w0(int, bool, bool, bool, bool);
+SweepFn lookup_sweep_w1(int, bool, bool, bool, bool);
+SweepFn lookup_sweep_w2(int, bool, bool, bool, bool);
+SweepFn lookup_sweep_w4(int, bool, bool, bool, bool);
+SweepFn lookup_sweep_w8(int, bool, bool, bool, bool);
+SweepFn lookup_sweep_w16(int, bool, bool, bool, bool);
+
+SweepFn lookup_sweep(int W, int gm, bool bf16, bool pre, bool step, bool post) {
+  switch (W) {
+    case 1: return lookup_sweep_w1(gm, bf16, pre, step, post);
+    case 2: return lookup_sweep_w2(gm, bf16, pre, step, post);
+    case 4: return lookup_sweep_w4(gm, bf16, pre, step, post);
+    case 8: return lookup_sweep_w8(gm, bf16, pre, step, post);
+    case 16: return lookup_sweep_w16(gm, bf16, pre, step, post);
+    default: return lookup_sweep_w0(gm, bf16, pre, step, post);
+  }
+}
+
+__global__ void la_fill(float* X, float* B2, float* Bs, const float* x0, float b0sq, uint64_t stride,
+                        uint64_t n, uint32_t W) {
+  const uint64_t nthreads = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < stride; j += nthreads) {
+    const float v = (x0 != nullptr && j < n) ? x0[j] : 0.0f;
+    for (uint32_t i = 0; i < W; ++i) {
+      X[(uint64_t)i * stride + j] = v;
+      B2[(uint64_t)i * stride + j] = b0sq;
+    }
+    Bs[j] = b0sq;
+  }
+}
+
+}  // namespace la
+
+namespace {
+
+thread_local std::string g_create_error;
+
+enum KernelClass { kClassLocal = 0, kClassSync = 1, kClassFused = 2, kClassOther = 3 };
+
+struct EventPair {
+  cudaEvent_t a, b;
+  int cls;
+};
+
+}  // namespace
+
+struct la_ctx {
+  // configuration
+  std::vector<uint64_t> sizes, offsets;
+  uint64_t N = 0, stride = 0, ngroups = 0, j_base = 0;
+  uint32_t W = 0, H = 0;
+  float eta = 0, eps = 0, b0sq = 0, sigma = 0;
+  uint32_t warm_up_steps = 0;
+  int grad_kind = la::kGradNoise;
+  bool bf16 = false, identical = false;
+  uint64_t seed = 0;
+  int fusion = LA_FUSE_NONE;
+  bool profiling = false;
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  int num_sms = 148;
+  int blocks_per_sm = 8;
+  // device memory
+  void* arena = nullptr;
+  bool owns_arena = false;
+  float *X = nullptr, *B2 = nullptr, *Bs = nullptr, *pa = nullptr, *pc = nullptr, *ps = nullptr;
+  bool has_s = false;
+  // schedule (Algorithm 3): t = local steps so far, tp = local steps since the last sync
+  uint64_t t = 0, nsync = 0;
+  uint32_t tp = 0;
+  // statistics
+  la_stats stats{};
+  std::vector<EventPair> pending;
+  std::vector<EventPair> pool;
+  std::string err;
+};
+
+namespace {
+
+int fail(la_ctx* c, int code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (c) c->err = buf; else g_create_error = buf;
+  return code;
+}
+
+#define LA_CUDA(ctx, call)                                                                      \
+  do {                                                                                          \
+    cudaError_t e_ = (call);                                                                    \
+    if (e_ != cudaSuccess) return fail((ctx), LA_ECUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+uint64_t round_up(uint64_t v, uint64_t m) { return (v + m - 1) / m * m; }
+
+// Layout of the arena, in floats: X[W][stride] | B2[W][stride] | Bs[stride] | a | c | s.
+// stride = N rounded up to 64 floats, so every sub-array starts on a 256-byte boundary and
+// the last group of four coordinates never leaves its array.
+int validate(const la_config* cfg, uint64_t* N_out) {
+  if (!cfg) return fail(nullptr, LA_EINVAL, "config is NULL");
+  if (cfg->K == 0 || cfg->sizes == nullptr) return fail(nullptr, LA_EINVAL, "K must be >= 1 and sizes non-NULL");
+  uint64_t N = 0;
+  for (uint32_t k = 0; k < cfg->K; ++k) {
+    if (cfg->sizes[k] == 0) return fail(nullptr, LA_EINVAL, "tensor %u has size 0", k);
+    if (N + cfg->sizes[k] < N) return fail(nullptr, LA_EINVAL, "total size overflows");
+    N += cfg->sizes[k];
+  }
+  if (N > (1ull << 40)) return fail(nullptr, LA_EINVAL, "N too large");
+  if (cfg->W == 0 || cfg->W > LA_MAX_WORKERS) return fail(nullptr, LA_EINVAL, "W must be in 1..%u", LA_MAX_WORKERS);
+  if (cfg->H == 0) return fail(nullptr, LA_EINVAL, "H must be >= 1");
+  if (!std::isfinite(cfg->eta)) return fail(nullptr, LA_EINVAL, "eta must be finite");
+  if (!(cfg->eps > 0.0f) || !std::isfinite(cfg->eps) || !(cfg->eps * cfg->eps > 0.0f))
+    return fail(nullptr, LA_EINVAL, "eps must be finite and eps*eps > 0 in fp32");
+  if (!(cfg->b0sq >= 0.0f) || !std::isfinite(cfg->b0sq)) return fail(nullptr, LA_EINVAL, "b0sq must be finite and >= 0");
+  if (cfg->j_base % 4 != 0) return fail(nullptr, LA_EINVAL, "j_base must be a multiple of 4");
+  *N_out = N;
+  return LA_OK;
+}
+
+uint64_t arena_floats(uint64_t N, uint32_t W) {
+  const uint64_t stride = round_up(N, 64);
+  return stride * (2ull * W + 4ull);
+}
+
+// ---- profiling events -------------------------------------------------------------------
+int drain_events(la_ctx* c) {
+  if (c->pending.empty()) return LA_OK;
+  LA_CUDA(c, cudaStreamSynchronize(c->stream));
+  for (auto& p : c->pending) {
+    float ms = 0.f;
+    LA_CUDA(c, cudaEventElapsedTime(&ms, p.a, p.b));
+    if (p.cls == kClassLocal) c->stats.ms_local += ms;
+    else if (p.cls == kClassSync) c->stats.ms_sync += ms;
+    else if (p.cls == kClassFused) c->stats.ms_fused += ms;
+    c->pool.push_back(p);
+  }
+  c->pending.clear();
+  return LA_OK;
+}
+
+int begin_timed(la_ctx* c, int cls, EventPair* ep) {
+  if (c->pending.size() >= 8192) {
+    int rc = drain_events(c);
+    if (rc) return rc;
+  }
+  if (!c->pool.empty()) {
+    *ep = c->pool.back();
+    c->pool.pop_back();
+  } else {
+    LA_CUDA(c, cudaEventCreate(&ep->a));
+    LA_CUDA(c, cudaEventCreate(&ep->b));
+  }
+  ep->cls = cls;
+  LA_CUDA(c, cudaEventRecord(ep->a, c->stream));
+  return LA_OK;
+}
+
+// ---- kernel dispatch ------------------------------------------------------------------------
+// Algorithmic bytes of one pass (what must cross HBM with the thread-per-coordinate mapping):
+// every replica's x and B^2 read and written once, worker-independent arrays once.
+double pass_bytes(const la_ctx* c, bool pre, bool step, bool post, int gm) {
+  const double n = (double)c->N, W = (double)c->W;
+  double b = 16.0 * W * n;                          // X, B2: read + write
+  if (pre || post) b += 4.0 * n;                    // stale accumulator written
+  if (step && !pre) b += 4.0 * n;                   // stale accumulator read
+  if (step) {
+    if (gm == la::kGradQuadratic) b += 8.0 * n;
+    if (gm == la::kGradNoiseScaled || (gm == la::kGradConstant && c->has_s)) b += 4.0 * n;
+    if (gm == la::kGradExternalF32) b += 4.0 * W * n;
+    if (gm == la::kGradExternalBF16) b += 2.0 * W * n;
+  }
+  return b;
+}
+
+int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t tp, int gm, const void* gext) {
+  la::SweepFn fn = la::lookup_sweep((int)c->W, gm, c->bf16 && gm <= la::kGradQuadratic, pre, step, post);
+  if (!fn) return fail(c, LA_ESTATE, "no kernel for this combination (W=%u grad=%d)", c->W, gm);
+  la::SweepParams p{};
+  p.X = c->X; p.B2 = c->B2; p.Bs = c->Bs;
+  p.a = c->pa; p.c = c->pc; p.s = c->has_s ? c->ps : nullptr;
+  p.gext = gext;
+  p.n = c->N; p.ngroups = c->ngroups; p.stride = c->stride; p.j_base = c->j_base;
+  p.seed = c->seed; p.t = t; p.W = c->W; p.tp = tp;
+  p.warm_up_steps = c->warm_up_steps; p.identical_workers = c->identical ? 1u : 0u;
+  p.eta = c->eta; p.eps = c->eps; p.sigma = c->sigma;
+  const unsigned block = 256;
+  uint64_t blocks = (c->ngroups + block - 1) / block;
+  const uint64_t cap = (uint64_t)c->num_sms * (uint64_t)c->blocks_per_sm;
+  if (blocks > cap) blocks = cap;
+  const int cls = (step && (pre || post)) ? kClassFused : (step ? kClassLocal : kClassSync);
+  EventPair ep{};
+  if (c->profiling) {
+    int rc = begin_timed(c, cls, &ep);
+    if (rc) return rc;
+  }
+  fn<<<(unsigned)blocks, block, 0, c->stream>>>(p);
+  LA_CUDA(c, cudaGetLastError());
+  if (c->profiling) {
+    LA_CUDA(c, cudaEventRecord(ep.b, c->stream));
+    c->pending.push_back(ep);
+  }
+  const double bytes = pass_bytes(c, pre, step, post, gm);
+  if (cls == kClassLocal) { c->stats.launches_local++; c->stats.bytes_local += bytes; }
+  else if (cls == kClassSync) { c->stats.launches_sync++; c->stats.bytes_sync += bytes; }
+  else { c->stats.launches_fused++; c->stats.bytes_fused += bytes; }
+  return LA_OK;
+}
+
+int upload_padded(la_ctx* c, float* dst, const float* src_host, float pad) {
+  // dst has `stride` floats; [0,N) from the host, the tail [N,stride) = pad.
+  LA_CUDA(c, cudaMemcpyAsync(dst, src_host, c->N * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+  if (c->stride > c->N) {
+    if (pad != 0.0f) return fail(c, LA_EINVAL, "internal: non-zero pad");
+    LA_CUDA(c, cudaMemsetAsync(dst + c->N, 0, (c->stride - c->N) * sizeof(float), c->stream));
+  }
+  return LA_OK;
+}
+
+int do_fill(la_ctx* c, const float* x0_dev) {
+  const unsigned block = 256;
+  uint64_t blocks = (c->stride + block - 1) / block;
+  const uint64_t cap = (uint64_t)c->num_sms * 16;
+  if (blocks > cap) blocks = cap;
+  la::la_fill<<<(unsigned)blocks, block, 0, c->stream>>>(c->X, c->B2, c->Bs, x0_dev, c->b0sq, c->stride, c->N, c->W);
+  LA_CUDA(c, cudaGetLastError());
+  c->stats.launches_other++;
+  return LA_OK;
+}
+
+}  // namespace
+
+// =============================================================================== C surface
+extern "C" {
+
+const char* la_last_error(const la_ctx* ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }
+
+int la_arena_bytes(const la_config* cfg, uint64_t* bytes) {
+  uint64_t N = 0;
+  int rc = validate(cfg, &N);
+  if (rc) return rc;
+  if (!bytes) return fail(nullptr, LA_EINVAL, "bytes is NULL");
+  *bytes = arena_floats(N, cfg->W) * sizeof(float);
+  return LA_OK;
+}
+
+int la_create_ex(la_ctx** out, const la_config* cfg) {
+  if (!out) return fail(nullptr, LA_EINVAL, "out is NULL");
+  *out = nullptr;
+  uint64_t N = 0;
+  int rc = validate(cfg, &N);
+  if (rc) return rc;
+  la_ctx* c = new (std::nothrow) la_ctx();
+  if (!c) return fail(nullptr, LA_ENOMEM, "host allocation failed");
+  auto bail = [&](int code, const char* what, cudaError_t e) {
+    fail(nullptr, code, "%s%s%s", what, e != cudaSuccess ? ": " : "", e != cudaSuccess ? cudaGetErrorString(e) : "");
+    if (c->owns_arena && c->arena) cudaFree(c->arena);
+    delete c;
+    return code;
+  };
+  cudaError_t e;
+  int dev = cfg->device;
+  if (dev < 0 && (e = cudaGetDevice(&dev)) != cudaSuccess) return bail(LA_ECUDA, "cudaGetDevice", e);
+  c->device = dev;
+  DeviceGuard guard(dev);
+  if (!guard.ok) return bail(LA_ECUDA, "cannot select device", cudaSuccess);
+  int sms = 0;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+    return bail(LA_ECUDA, "cudaDeviceGetAttribute", e);
+  c->num_sms = sms > 0 ? sms : 148;
+  c->sizes.assign(cfg->sizes, cfg->sizes + cfg->K);
+  c->offsets.resize(cfg->K);
+  uint64_t off = 0;
+  for (uint32_t k = 0; k < cfg->K; ++k) { c->offsets[k] = off; off += c->sizes[k]; }
+  c->N = N;
+  c->stride = round_up(N, 64);
+  c->ngroups = (N + 3) / 4;
+  c->j_base = cfg->j_base;
+  c->W = cfg->W; c->H = cfg->H; c->eta = cfg->eta; c->eps = cfg->eps; c->b0sq = cfg->b0sq;
+  c->stream = (cudaStream_t)cfg->stream;
+  const uint64_t need = arena_floats(N, cfg->W) * sizeof(float);
+  if (cfg->dev_arena) {
+    if (cfg->arena_bytes < need) return bail(LA_ENOMEM, "caller arena smaller than la_arena_bytes()", cudaSuccess);
+    if (((uintptr_t)cfg->dev_arena & 255u) != 0) return bail(LA_EINVAL, "caller arena must be 256-byte aligned", cudaSuccess);
+    c->arena = cfg->dev_arena;
+  } else {
+    if ((e = cudaMalloc(&c->arena, need)) != cudaSuccess) {
+      c->arena = nullptr;
+      cudaGetLastError();
+      return bail(LA_ENOMEM, "cudaMalloc of the state arena failed", e);
+    }
+    c->owns_arena = true;
+  }
+  float* base = (float*)c->arena;
+  c->X = base;
+  c->B2 = c->X + (uint64_t)c->W * c->stride;
+  c->Bs = c->B2 + (uint64_t)c->W * c->stride;
+  c->pa = c->Bs + c->stride;
+  c->pc = c->pa + c->stride;
+  c->ps = c->pc + c->stride;
+  // problem arrays start as zeros so that padded coordinates stay finite in every mode
+  if ((e = cudaMemsetAsync(c->pa, 0, 3 * c->stride * sizeof(float), c->stream)) != cudaSuccess)
+    return bail(LA_ECUDA, "cudaMemsetAsync", e);
+  c->grad_kind = la::kGradNoise;
+  rc = do_fill(c, nullptr);
+  if (rc) { g_create_error = c->err; if (c->owns_arena) cudaFree(c->arena); delete c; return rc; }
+  *out = c;
+  return LA_OK;
+}
+
+int la_create(la_ctx** out, uint64_t N, uint32_t W, float eta, float eps, uint32_t H) {
+  la_config cfg;
+  std::memset(&cfg, 0, sizeof cfg);
+  cfg.K = 1; cfg.sizes = &N; cfg.W = W; cfg.H = H; cfg.eta = eta; cfg.eps = eps; cfg.b0sq = 0.0f;
+  cfg.device = -1;
+  return la_create_ex(out, &cfg);
+}
+
+void la_destroy(la_ctx* c) {
+  if (!c) return;
+  DeviceGuard guard(c->device);
+  cudaStreamSynchronize(c->stream);
+  for (auto& p : c->pending) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
+  for (auto& p : c->pool) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
+  if (c->owns_arena && c->arena) cudaFree(c->arena);
+  delete c;
+}
+
+int la_set_init(la_ctx* c, const float* x0_host, float b0sq) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!(b0sq >= 0.0f) || !std::isfinite(b0sq)) return fail(c, LA_EINVAL, "b0sq must be finite and >= 0");
+  DeviceGuard guard(c->device);
+  c->b0sq = b0sq;
+  const float* x0_dev = nullptr;
+  if (x0_host) {
+    // stage x0 in replica 0's own slot, then broadcast from there
+    LA_CUDA(c, cudaMemcpyAsync(c->X, x0_host, c->N * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+    x0_dev = c->X;
+  }
+  int rc = do_fill(c, x0_dev);
+  if (rc) return rc;
+  c->t = 0; c->tp = 0; c->nsync = 0;
+  return LA_OK;
+}
+
+int la_set_grad_noise(la_ctx* c, uint64_t seed, const float* s_host) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  DeviceGuard guard(c->device);
+  c->seed = seed;
+  c->has_s = s_host != nullptr;
+  c->grad_kind = s_host ? la::kGradNoiseScaled : la::kGradNoise;
+  if (s_host) return upload_padded(c, c->ps, s_host, 0.0f);
+  return LA_OK;
+}
+
+int la_set_grad_quadratic(la_ctx* c, uint64_t seed, const float* a_host, const float* c_host, float sigma) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!a_host || !c_host) return fail(c, LA_EINVAL, "a and c must be non-NULL");
+  if (!std::isfinite(sigma)) return fail(c, LA_EINVAL, "sigma must be finite");
+  DeviceGuard guard(c->device);
+  c->seed = seed; c->sigma = sigma; c->grad_kind = la::kGradQuadratic;
+  int rc = upload_padded(c, c->pa, a_host, 0.0f);
+  if (rc) return rc;
+  return upload_padded(c, c->pc, c_host, 0.0f);
+}
+
+int la_set_grad_constant(la_ctx* c, const float* s_host) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  DeviceGuard guard(c->device);
+  c->grad_kind = la::kGradConstant;
+  c->has_s = s_host != nullptr;
+  if (s_host) return upload_padded(c, c->ps, s_host, 0.0f);
+  return LA_OK;
+}
+
+int la_set_grad_dtype(la_ctx* c, int dtype) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (dtype != LA_F32 && dtype != LA_BF16) return fail(c, LA_EINVAL, "dtype must be LA_F32 or LA_BF16");
+  c->bf16 = dtype == LA_BF16;
+  return LA_OK;
+}
+
+int la_set_identical_workers(la_ctx* c, int on) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  c->identical = on != 0;
+  return LA_OK;
+}
+
+int la_set_warmup(la_ctx* c, uint32_t steps) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  c->warm_up_steps = steps;
+  return LA_OK;
+}
+
+int la_set_fusion(la_ctx* c, int mode) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (mode != LA_FUSE_NONE && mode != LA_FUSE_STEP_SYNC && mode != LA_FUSE_SYNC_STEP)
+    return fail(c, LA_EINVAL, "unknown fusion mode %d", mode);
+  c->fusion = mode;
+  return LA_OK;
+}
+
+int la_set_profiling(la_ctx* c, int on) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  DeviceGuard guard(c->device);
+  if (!on) { int rc = drain_events(c); if (rc) return rc; }
+  c->profiling = on != 0;
+  return LA_OK;
+}
+
+int la_set_launch_shape(la_ctx* c, int blocks_per_sm) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (blocks_per_sm < 1 || blocks_per_sm > 4096) return fail(c, LA_EINVAL, "blocks_per_sm out of range");
+  c->blocks_per_sm = blocks_per_sm;
+  return LA_OK;
+}
+
+// ---- hot path ------------------------------------------------------------------------------
+int la_local_step(la_ctx* c) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  DeviceGuard guard(c->device);
+  int rc = launch_sweep(c, false, true, false, c->t + 1, c->tp + 1, c->grad_kind, nullptr);
+  if (rc) return rc;
+  c->t += 1; c->tp += 1;
+  return LA_OK;
+}
+
+int la_local_step_grads(la_ctx* c, const void* g_dev, int dtype) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!g_dev) return fail(c, LA_EINVAL, "g_dev is NULL");
+  if (dtype != LA_F32 && dtype != LA_BF16) return fail(c, LA_EINVAL, "dtype must be LA_F32 or LA_BF16");
+  DeviceGuard guard(c->device);
+  int rc = launch_sweep(c, false, true, false, c->t + 1, c->tp + 1,
+                        dtype == LA_F32 ? la::kGradExternalF32 : la::kGradExternalBF16, g_dev);
+  if (rc) return rc;
+  c->t += 1; c->tp += 1;
+  return LA_OK;
+}
+
+int la_sync(la_ctx* c) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  DeviceGuard guard(c->device);
+  int rc = launch_sweep(c, true, false, false, c->t, 0, la::kGradNoise, nullptr);
+  if (rc) return rc;
+  c->tp = 0; c->nsync += 1;
+  return LA_OK;
+}
+
+int la_run(la_ctx* c, uint64_t T) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  DeviceGuard guard(c->device);
+  // Algorithm 3: for t in [T]: local step; if mod(t, H) == 0 (tracked as t' == H): synchronise.
+  // `deferred` marks a synchronisation that is due but has been folded into the next step.
+  bool deferred = false;
+  for (uint64_t k = 0; k < T; ++k) {
+    int rc;
+    if (deferred) {
+      rc = launch_sweep(c, true, true, false, c->t + 1, 1, c->grad_kind, nullptr);  // K4: sync, then step t'=1
+      if (rc) return rc;
+      c->nsync += 1; c->t += 1; c->tp = 1;
+      deferred = false;
+    } else if (c->fusion == LA_FUSE_STEP_SYNC && c->tp + 1 == c->H) {
+      rc = launch_sweep(c, false, true, true, c->t + 1, c->tp + 1, c->grad_kind, nullptr);  // K3: step t'=H and its sync
+      if (rc) return rc;
+      c->t += 1; c->tp = 0; c->nsync += 1;
+      continue;
+    } else {
+      rc = la_local_step(c);  // K1
+      if (rc) return rc;
+    }
+    if (c->tp == c->H) {
+      if (c->fusion == LA_FUSE_SYNC_STEP && k + 1 < T) {
+        deferred = true;
+      } else {
+        rc = la_sync(c);  // K2
+        if (rc) return rc;
+      }
+    }
+  }
+  return LA_OK;
+}
+
+// ---- state access ----------------------------------------------------------------------------
+int la_read_range(la_ctx* c, uint32_t worker, uint64_t j0, uint64_t n, float* x_host, float* b2_host, float* bs_host) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (worker >= c->W) return fail(c, LA_EINVAL, "worker %u out of range (W=%u)", worker, c->W);
+  if (j0 > c->N || n > c->N - j0) return fail(c, LA_EINVAL, "coordinate range out of bounds");
+  DeviceGuard guard(c->device);
+  const size_t bytes = n * sizeof(float);
+  if (n) {
+    if (x_host) LA_CUDA(c, cudaMemcpyAsync(x_host, c->X + (uint64_t)worker * c->stride + j0, bytes, cudaMemcpyDeviceToHost, c->stream));
+    if (b2_host) LA_CUDA(c, cudaMemcpyAsync(b2_host, c->B2 + (uint64_t)worker * c->stride + j0, bytes, cudaMemcpyDeviceToHost, c->stream));
+    if (bs_host) LA_CUDA(c, cudaMemcpyAsync(bs_host, c->Bs + j0, bytes, cudaMemcpyDeviceToHost, c->stream));
+  }
+  LA_CUDA(c, cudaStreamSynchronize(c->stream));
+  return LA_OK;
+}
+
+int la_read_state(la_ctx* c, uint32_t worker, float* x_host, float* b2_host, float* bs_host) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  return la_read_range(c, worker, 0, c->N, x_host, b2_host, bs_host);
+}
+
+int la_write_state(la_ctx* c, uint32_t worker, const float* x_host, const float* b2_host, const float* bs_host) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (worker >= c->W) return fail(c, LA_EINVAL, "worker %u out of range (W=%u)", worker, c->W);
+  DeviceGuard guard(c->device);
+  const size_t bytes = c->N * sizeof(float);
+  if (x_host) LA_CUDA(c, cudaMemcpyAsync(c->X + (uint64_t)worker * c->stride, x_host, bytes, cudaMemcpyHostToDevice, c->stream));
+  if (b2_host) LA_CUDA(c, cudaMemcpyAsync(c->B2 + (uint64_t)worker * c->stride, b2_host, bytes, cudaMemcpyHostToDevice, c->stream));
+  if (bs_host) LA_CUDA(c, cudaMemcpyAsync(c->Bs, bs_host, bytes, cudaMemcpyHostToDevice, c->stream));
+  LA_CUDA(c, cudaStreamSynchronize(c->stream));
+  return LA_OK;
+}
+
+int la_tensor_range(const la_ctx* c, uint32_t k, uint64_t* offset, uint64_t* size) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (k >= c->sizes.size()) return fail(const_cast<la_ctx*>(c), LA_EINVAL, "tensor %u out of range", k);
+  if (offset) *offset = c->offsets[k];
+  if (size) *size = c->sizes[k];
+  return LA_OK;
+}
+
+int la_get_counters(const la_ctx* c, uint64_t* t, uint32_t* t_prime, uint64_t* n_sync) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (t) *t = c->t;
+  if (t_prime) *t_prime = c->tp;
+  if (n_sync) *n_sync = c->nsync;
+  return LA_OK;
+}
+
+int la_set_counters(la_ctx* c, uint64_t t, uint32_t t_prime, uint64_t n_sync) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  c->t = t; c->tp = t_prime; c->nsync = n_sync;
+  return LA_OK;
+}
+
+int la_get_stats(la_ctx* c, la_stats* out, int reset) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!out) return fail(c, LA_EINVAL, "out is NULL");
+  DeviceGuard guard(c->device);
+  int rc = drain_events(c);
+  if (rc) return rc;
+  *out = c->stats;
+  if (reset) c->stats = la_stats{};
+  return LA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,318 @@
+"""GPU parity: the CUDA library (through its C-ABI) against the CPU oracle, element by
+element on the same seeded inputs.  Contract: |gpu - ref| <= 1e-6 max(1,|ref|) after one
+step and <= 1e-5 max(1,|ref|) after a full run; counters bit-exact.  Because both sides
+perform the same sequence of correctly rounded fp32 operations the tests also demand
+bitwise equality."""
+import itertools
+
+import numpy as np
+import pytest
+
+from oracle.oracle import Oracle
+from paper_1911_09030_b200 import local_adaalter as la
+from paper_1911_09030_b200 import workloads
+from parity_util import compare, make_pair
+
+pytestmark = pytest.mark.gpu
+
+TOL_STEP, TOL_RUN = 1e-6, 1e-5
+
+
+def _arrays(n, seed):
+    rng = np.random.default_rng(seed)
+    return dict(a=rng.uniform(0.1, 10, n).astype(np.float32), c=rng.standard_normal(n).astype(np.float32),
+                s=np.exp(rng.uniform(np.log(1e-3), 0, n)).astype(np.float32))
+
+
+# ----------------------------------------------------------------------------- configuration 1
+@pytest.mark.parametrize("fusion", [0, 1, 2])
+def test_config1_full(fusion):
+    wl = workloads.config("c1")
+    arr = wl.arrays()
+    g, o = make_pair(wl.N, wl.W, wl.eta, wl.eps, wl.H, "quadratic", seed=wl.noise_seed, arrays=arr,
+                     sigma=wl.sigma, fusion=fusion)
+    g.run(1)
+    o.run(1)
+    compare(g, o, wl.W, TOL_STEP)
+    g.run(wl.T - 1)
+    o.run(wl.T - 1)
+    compare(g, o, wl.W, TOL_RUN)
+    assert g.get_counters() == (wl.T, 0, wl.T // wl.H)
+
+
+# ----------------------------------------------------------------------------- shape sweep
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 31, 32, 33, 1023, 1025])
+@pytest.mark.parametrize("W", [1, 2, 3, 4, 8, 16])
+def test_tails_and_worker_counts(n, W):
+    T = 7
+    arr = _arrays(n, 10 * n + W)
+    for H, grad, fusion in [(1, "quadratic", 0), (2, "noise_scaled", 1), (3, "quadratic", 2), (T, "noise", 1),
+                            (T + 1, "quadratic", 2)]:
+        g, o = make_pair(n, W, 0.1, 0.5, H, grad, seed=n + W, arrays=arr, sigma=0.3, fusion=fusion, b0sq=0.25)
+        g.run(T)
+        o.run(T)
+        compare(g, o, W, TOL_RUN)
+        g.close()
+
+
+@pytest.mark.parametrize("W", [5, 6, 7, 11, 13, 64])
+def test_generic_worker_counts(W):
+    n, T = 257, 9
+    arr = _arrays(n, W)
+    for H, fusion in [(2, 0), (3, 1), (4, 2)]:
+        g, o = make_pair(n, W, 0.05, 1.0, H, "quadratic", seed=W, arrays=arr, sigma=1.0, fusion=fusion)
+        g.run(T)
+        o.run(T)
+        compare(g, o, W, TOL_RUN)
+
+
+@pytest.mark.parametrize("grad,bf16", [("noise", False), ("noise", True), ("noise_scaled", False),
+                                       ("noise_scaled", True), ("quadratic", False), ("quadratic", True),
+                                       ("constant", False)])
+@pytest.mark.parametrize("fusion", [0, 1, 2])
+def test_gradient_modes(grad, bf16, fusion):
+    n, W, H, T = 70001, 4, 3, 10      # several blocks and a ragged tail
+    arr = _arrays(n, 3)
+    g, o = make_pair(n, W, 0.05, 0.7, H, grad, seed=21, arrays=arr, sigma=0.5, bf16=bf16, fusion=fusion)
+    g.run(1)
+    o.run(1)
+    compare(g, o, W, TOL_STEP)
+    g.run(T - 1)
+    o.run(T - 1)
+    compare(g, o, W, TOL_RUN)
+
+
+# ----------------------------------------------------------------------------- fused == unfused
+@pytest.mark.parametrize("W,H", [(2, 1), (4, 4), (8, 3), (16, 2), (3, 2)])
+def test_fused_kernels_equal_unfused_bitwise(W, H):
+    n, T = 12345, 11
+    arr = _arrays(n, 77)
+    states = []
+    for fusion in (0, 1, 2):
+        g = la.LocalAdaAlter([n], W, 0.1, 1.0, H)
+        g.set_grad_quadratic(5, arr["a"], arr["c"], 0.2)
+        g.set_fusion(fusion)
+        g.run(4)
+        g.run(T - 4)                   # a run boundary in the middle of a period
+        states.append(([g.read_state(i) for i in range(W)], g.get_counters(), g.get_stats()))
+        g.close()
+    for st, cnt, stats in states[1:]:
+        assert cnt == states[0][1]
+        for i in range(W):
+            for u, v in zip(st[i], states[0][0][i]):
+                assert np.array_equal(u.view(np.uint32), v.view(np.uint32))
+    assert states[0][2]["launches_fused"] == 0 and states[0][2]["launches_sync"] == T // H
+    assert states[1][2]["launches_fused"] == T // H and states[1][2]["launches_sync"] == 0
+    assert states[2][2]["launches_fused"] > 0
+
+
+# ----------------------------------------------------------------------------- schedule
+@pytest.mark.parametrize("H,T", [(1, 5), (2, 5), (3, 9), (5, 5), (6, 5), (la.LA_H_NEVER, 6)])
+@pytest.mark.parametrize("fusion", [0, 1, 2])
+def test_schedule_counters_match_oracle(H, T, fusion):
+    g, o = make_pair(64, 2, 0.1, 1.0, H, "noise", seed=1, fusion=fusion)
+    for _ in range(T):
+        g.run(1)
+        o.run(1)
+        assert g.get_counters() == o.counters()
+    compare(g, o, 2, TOL_RUN)
+
+
+def test_manual_steps_and_sync():
+    g, o = make_pair(100, 4, 0.2, 1.0, 10, "noise", seed=3)
+    for k in range(3):
+        g.local_step(); o.local_step()
+    g.sync(); o.sync()
+    g.local_step(); o.local_step()
+    g.sync(); o.sync()
+    g.sync(); o.sync()
+    compare(g, o, 4, TOL_RUN)
+    assert g.get_counters() == (4, 0, 3)
+
+
+def test_warmup_matches_oracle():
+    g, o = make_pair(513, 4, 0.5, 1.0, 4, "noise", seed=8, warmup=6, b0sq=1.0)
+    g.run(11); o.run(11)
+    compare(g, o, 4, TOL_RUN)
+
+
+def test_initial_iterate_and_b0():
+    n = 777
+    x0 = np.random.default_rng(0).standard_normal(n).astype(np.float32)
+    arr = _arrays(n, 1)
+    g, o = make_pair(n, 8, 0.5, 1.0, 4, "quadratic", seed=2, arrays=arr, sigma=1.0, x0=x0, b0sq=1.0, fusion=2)
+    g.run(9); o.run(9)
+    compare(g, o, 8, TOL_RUN)
+
+
+# ----------------------------------------------------------------------------- invariants on the GPU
+def test_identical_workers_stay_bitwise_equal():
+    n, W = 4099, 8
+    arr = _arrays(n, 5)
+    g, o = make_pair(n, W, 0.1, 1.0, 4, "quadratic", seed=9, arrays=arr, sigma=0.1, identical=True, fusion=1)
+    g.run(10); o.run(10)
+    compare(g, o, W, TOL_RUN)
+    x0, b0, _ = g.read_state(0)
+    for i in range(1, W):
+        x, b, _ = g.read_state(i)
+        assert np.array_equal(x, x0) and np.array_equal(b, b0)
+
+
+def test_constant_gradient_closed_form_on_gpu():
+    """B^2 = b0^2 + k g^2 and x_T from the closed form, independent of the oracle."""
+    n, W, H, T = 6, 4, 3, 23
+    gvec = np.array([0.5, -1.5, 2.0, 1.0, -0.25, 3.0], np.float32)
+    eta, eps, b0sq = 0.5, 0.75, 1.0
+    g = la.LocalAdaAlter([n], W, eta, eps, H, b0sq=b0sq)
+    g.set_init(None, b0sq)
+    g.set_grad_constant(gvec)
+    g.run(T)
+    exp_x = np.zeros(n)
+    for t in range(1, T + 1):
+        tp = (t - 1) % H + 1
+        exp_x -= eta * gvec.astype(np.float64) / np.sqrt(b0sq + (t - tp) * gvec.astype(np.float64) ** 2 + tp * eps * eps)
+    for i in range(W):
+        x, b2, bs = g.read_state(i)
+        np.testing.assert_allclose(b2, b0sq + T * gvec.astype(np.float64) ** 2, rtol=1e-6)
+        np.testing.assert_allclose(x, exp_x, rtol=5e-6)
+        np.testing.assert_allclose(bs, b0sq + (T - T % H) * gvec.astype(np.float64) ** 2, rtol=1e-6)
+
+
+def test_hand_worked_case_with_supplied_gradients():
+    """The hand-derived Algorithm-3 trajectory, driven through la_local_step_grads."""
+    import os
+    import torch
+    rows = [[float(v) for v in l.split()] for l in
+            open(os.path.join(os.path.dirname(__file__), "golden", "alg3_hand_case.txt"))
+            if l.strip() and not l.startswith("#")]
+    g = la.LocalAdaAlter([1], 2, 1.0, 1.0, 2)
+    for t, g0, g1, x0, x1, b0, b1, bs in rows:
+        grads = torch.tensor([[g0], [g1]], dtype=torch.float32, device="cuda")
+        g.local_step_grads(grads.data_ptr(), la.LA_F32)
+        if g.get_counters()[1] == 2:
+            g.sync()
+        xa, ba, sa = g.read_state(0)
+        xb, bb, _ = g.read_state(1)
+        assert xa[0] == pytest.approx(x0, abs=5e-7) and xb[0] == pytest.approx(x1, abs=5e-7)
+        assert (ba[0], bb[0], sa[0]) == (b0, b1, bs)
+    assert g.get_counters() == (4, 0, 2)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("n", [5, 64, 1001])
+def test_supplied_gradients_match_oracle(dtype, n):
+    import torch
+    W, H, T = 3, 2, 5
+    rng = np.random.default_rng(n)
+    g = la.LocalAdaAlter([n], W, 0.3, 0.5, H, b0sq=0.25)
+    g.set_init(None, 0.25)
+    o = Oracle(n, W, 0.3, 0.5, H, 0.25)
+    for t in range(T):
+        G = torch.from_numpy(rng.standard_normal((W, n)).astype(np.float32))
+        if dtype == "bf16":
+            Gd = G.to(torch.bfloat16).cuda()
+            g.local_step_grads(Gd.data_ptr(), la.LA_BF16)
+            o.local_step(Gd.float().cpu().numpy())
+        else:
+            Gd = G.cuda()
+            g.local_step_grads(Gd.data_ptr(), la.LA_F32)
+            o.local_step(G.numpy())
+        if g.get_counters()[1] == H:
+            g.sync(); o.sync()
+        g.sync_stream()
+    compare(g, o, W, TOL_RUN)
+
+
+def test_checkpoint_resume_bitwise():
+    n, W, H = 3001, 4, 4
+    arr = _arrays(n, 6)
+
+    def make():
+        c = la.LocalAdaAlter([n], W, 0.1, 1.0, H)
+        c.set_grad_quadratic(7, arr["a"], arr["c"], 0.1)
+        c.set_fusion(2)
+        return c
+
+    whole = make(); whole.run(11)
+    first = make(); first.run(6)
+    second = make()
+    for i in range(W):
+        x, b2, bs = first.read_state(i)
+        second.write_state(i, x, b2, bs)
+    second.set_counters(*first.get_counters())
+    second.run(5)
+    assert whole.get_counters() == second.get_counters() == (11, 3, 2)
+    for i in range(W):
+        for u, v in zip(whole.read_state(i), second.read_state(i)):
+            assert np.array_equal(u.view(np.uint32), v.view(np.uint32))
+
+
+def test_coordinate_sharding_is_exact():
+    """Two contexts that own the halves of the coordinate range reproduce the whole job."""
+    n, W = 4096 + 512, 4
+    arr = _arrays(n, 12)
+    whole = la.LocalAdaAlter([n], W, 0.01, 1e-3, 8)
+    whole.set_grad_noise(2, arr["s"]); whole.run(20)
+    cut = 2048
+    parts = []
+    for lo, hi in ((0, cut), (cut, n)):
+        p = la.LocalAdaAlter([hi - lo], W, 0.01, 1e-3, 8, j_base=lo)
+        p.set_grad_noise(2, arr["s"][lo:hi]); p.run(20)
+        parts.append(p)
+    for i in range(W):
+        full = whole.read_state(i)
+        for k in range(3):
+            joined = np.concatenate([parts[0].read_state(i)[k], parts[1].read_state(i)[k]])
+            assert np.array_equal(joined.view(np.uint32), full[k].view(np.uint32))
+
+
+def test_multi_tensor_views_and_torch_arena():
+    import torch
+    sizes = [1000, 3, 4096, 77]
+    n = sum(sizes)
+    arr = _arrays(n, 4)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        g = la.LocalAdaAlter.with_torch_arena(sizes, 4, 0.1, 1.0, 4)
+        g.set_grad_quadratic(3, arr["a"], arr["c"], 0.5)
+        g.run(9)
+    o = Oracle(n, 4, 0.1, 1.0, 4)
+    o.set_grad_quadratic(3, arr["a"], arr["c"], 0.5)
+    o.run(9)
+    compare(g, o, 4, TOL_RUN)
+    off = 0
+    for k, sz in enumerate(sizes):
+        assert g.tensor_range(k) == (off, sz)
+        off += sz
+
+
+def test_runtime_errors_are_reported_not_fatal():
+    g = la.LocalAdaAlter([64], 2, 0.1, 1.0, 2)
+    with pytest.raises(la.LocalAdaAlterError) as e:
+        g.read_state(5)
+    assert e.value.code == la.LA_EINVAL and "worker" in str(e.value)
+    with pytest.raises(la.LocalAdaAlterError):
+        g.read_range(0, 60, 10)
+    with pytest.raises(la.LocalAdaAlterError):
+        g.set_fusion(9)
+    with pytest.raises(la.LocalAdaAlterError):
+        g.local_step_grads(0)
+    g.run(3)                                   # the context is still usable
+    assert g.get_counters() == (3, 1, 1)
+    import torch
+    too_small = torch.empty(16, device="cuda")
+    with pytest.raises(la.LocalAdaAlterError) as e:
+        la.LocalAdaAlter([64], 2, 0.1, 1.0, 2, arena=too_small)
+    assert e.value.code == la.LA_ENOMEM
+
+
+def test_profiling_stats():
+    g = la.LocalAdaAlter([1 << 16], 4, 0.1, 1.0, 4)
+    g.set_grad_noise(1)
+    g.set_profiling(True)
+    g.run(8)
+    st = g.get_stats()
+    assert st["launches_local"] == 8 and st["launches_sync"] == 2
+    assert st["ms_local"] > 0 and st["ms_sync"] > 0
+    assert st["bytes_local"] == 8 * (16 * 4 + 4) * (1 << 16)
+    assert st["bytes_sync"] == 2 * (16 * 4 + 4) * (1 << 16)
