@@ -28,6 +28,23 @@ import numpy as np
 METRIC = "worker_param_updates_per_sec"
 UNIT = "worker*param updates/s"
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from
+# the ncu capture summarised in profiles/), valid only for the kernel sources they were taken on.
+KERNEL_HASH_AT_CAPTURE = "489667179e4edd72"
+NCU_TRAFFIC_BYTES = {"c2": 2.2238e9}
+
+
+def kernel_source_hash():
+    import glob
+    import hashlib
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_1911_09030_b200", "csrc")
+    for pat in ("*.cu", "*.cuh", "*.inc"):
+        for f in sorted(glob.glob(os.path.join(d, pat))):
+            with open(f, "rb") as fh:
+                h.update(fh.read())
+    return h.hexdigest()[:16]
 
 
 def measured_peak():
@@ -263,7 +280,10 @@ def run_ours(args, wl):
         roofline = {
             "bound": "hbm", "kernel": "la_sweep<STEP> (K1 local step)", "achieved": achieved, "peak": peak,
             "peak_kind": peak_kind, "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
-            "traffic": None, "bytes_per_launch": bytes_local, "ms_per_launch": ms_local,
+            "traffic": (NCU_TRAFFIC_BYTES.get(wl.name) if kernel_source_hash() == KERNEL_HASH_AT_CAPTURE
+                        and args.H is None else None),
+            "frac_of_nominal_8TBps": (achieved / NOMINAL_HBM_GBS) if achieved else None,
+            "bytes_per_launch": bytes_local, "ms_per_launch": ms_local,
             "bytes_per_update": bytes_local / (wl.W * wl.N),
         }
         per_class = {}

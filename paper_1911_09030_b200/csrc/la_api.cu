@@ -77,7 +77,7 @@ struct la_ctx {
   int device = 0;
   cudaStream_t stream = nullptr;
   int num_sms = 148;
-  int blocks_per_sm = 8;
+  int blocks_per_sm = 0;  // 0 = per-kernel default
   // device memory
   void* arena = nullptr;
   bool owns_arena = false;
@@ -216,9 +216,14 @@ int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t
   p.seed = c->seed; p.t = t; p.W = c->W; p.tp = tp;
   p.warm_up_steps = c->warm_up_steps; p.identical_workers = c->identical ? 1u : 0u;
   p.eta = c->eta; p.eps = c->eps; p.sigma = c->sigma;
-  const unsigned block = 256;
+  const unsigned block = la::kBlockThreads;
   uint64_t blocks = (c->ngroups + block - 1) / block;
-  const uint64_t cap = (uint64_t)c->num_sms * (uint64_t)c->blocks_per_sm;
+  // Measured on B200: kernels that generate gradients run best with about 48 blocks per SM in
+  // the grid (each thread then handles a few coordinate groups, so the software pipeline pays
+  // off, while blocks are still small enough to balance the SMs); the pure averaging kernel
+  // runs best with one group per thread.
+  const int bps = c->blocks_per_sm > 0 ? c->blocks_per_sm : (step ? 48 : 4096);
+  const uint64_t cap = (uint64_t)c->num_sms * (uint64_t)bps;
   if (blocks > cap) blocks = cap;
   const int cls = (step && (pre || post)) ? kClassFused : (step ? kClassLocal : kClassSync);
   EventPair ep{};
@@ -442,7 +447,7 @@ int la_set_profiling(la_ctx* c, int on) {
 
 int la_set_launch_shape(la_ctx* c, int blocks_per_sm) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
-  if (blocks_per_sm < 1 || blocks_per_sm > 4096) return fail(c, LA_EINVAL, "blocks_per_sm out of range");
+  if (blocks_per_sm < 0 || blocks_per_sm > 4096) return fail(c, LA_EINVAL, "blocks_per_sm out of range");
   c->blocks_per_sm = blocks_per_sm;
   return LA_OK;
 }

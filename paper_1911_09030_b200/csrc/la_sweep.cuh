@@ -102,15 +102,55 @@ struct PairTree {
   }
 };
 
-template <int GM>
-struct GradInputs {
-  float4 a, c, s;
+// Worker-independent data of one coordinate group: the stale accumulator and the problem arrays.
+struct CoordInputs {
+  float4 bs, a, c, s;
 };
+
+template <int GM, bool STEP, bool LOAD_BS>
+__device__ __forceinline__ void load_coord(CoordInputs& in, const SweepParams& p, uint64_t off) {
+  if (LOAD_BS) in.bs = ld_stream(p.Bs + off);
+  if (STEP) {
+    if (GM == kGradQuadratic) {
+      in.a = ld_stream(p.a + off);
+      in.c = ld_stream(p.c + off);
+    }
+    if (GM == kGradNoiseScaled) in.s = ld_stream(p.s + off);
+    if (GM == kGradConstant) in.s = p.s ? ld_stream(p.s + off) : make_float4(1.f, 1.f, 1.f, 1.f);
+  }
+}
+
+// x and B^2 of CH consecutive replicas for one coordinate group.
+template <int CH>
+struct ReplicaChunk {
+  float4 x[CH], b[CH];
+};
+
+template <int CH>
+__device__ __forceinline__ void load_chunk(ReplicaChunk<CH>& ch, const SweepParams& p, uint32_t W, uint32_t i0,
+                                           uint64_t off) {
+#pragma unroll
+  for (int k = 0; k < CH; ++k)
+    if (i0 + k < W) {
+      ch.x[k] = ld_stream(p.X + (uint64_t)(i0 + k) * p.stride + off);
+      ch.b[k] = ld_stream(p.B2 + (uint64_t)(i0 + k) * p.stride + off);
+    }
+}
+
+// r = eta_t / sqrt(B^2_{t-t'} + t' eps^2): the step size all workers share (Section 4.2).
+__device__ __forceinline__ float4 step_size(float4 bs, float q, float eta_t) {
+  float4 r;
+  r.x = __fdiv_rn(eta_t, __fsqrt_rn(__fadd_rn(bs.x, q)));
+  r.y = __fdiv_rn(eta_t, __fsqrt_rn(__fadd_rn(bs.y, q)));
+  r.z = __fdiv_rn(eta_t, __fsqrt_rn(__fadd_rn(bs.z, q)));
+  r.w = __fdiv_rn(eta_t, __fsqrt_rn(__fadd_rn(bs.w, q)));
+  return r;
+}
 
 // Gradient of four coordinates for one worker.  `xv` is the worker's own iterate
 // (Algorithm 3: G_{i,t} = grad f(x_{i,t-1}; z_{i,t})).
 template <int GM, bool BF16>
-__device__ __forceinline__ float4 gradient4(const SweepParams& p, const GradInputs<GM>& in, float4 xv,
+__device__ __forceinline__ float4 gradient4(const SweepParams& p, const CoordInputs& in, float4 xv,
                                             uint64_t key, uint64_t ctr0, uint32_t worker, uint64_t off) {
   float4 g;
   if (GM == kGradConstant) {
@@ -168,11 +208,21 @@ __device__ __forceinline__ void apply4(float4 r, float4 g, float4& x, float4& b)
   b.w = __fmaf_rn(g.w, g.w, b.w);
 }
 
+#ifndef LA_BLOCK
+#define LA_BLOCK 256
+#endif
+#ifndef LA_CH
+#define LA_CH 4
+#endif
+constexpr int kBlockThreads = LA_BLOCK;
+
 template <int W_, int GM, bool BF16, bool PRE, bool STEP, bool POST, int MINB>
-__global__ void __launch_bounds__(256, MINB) la_sweep(const SweepParams p) {
+__global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) {
   static_assert(!(PRE && POST), "one synchronisation per pass");
   constexpr bool kNeedsNoise = STEP && (GM == kGradNoise || GM == kGradNoiseScaled || GM == kGradQuadratic);
-  constexpr int CH = (W_ > 0) ? (W_ < 8 ? W_ : 8) : 4;  // replicas loaded before any is consumed
+  constexpr int CH = (W_ > 0) ? (W_ < LA_CH ? W_ : LA_CH) : 4;  // replicas loaded before any is consumed
+  constexpr int kOuterUnroll = (W_ > 0) ? kMaxWorkers : 1;  // static W: unroll fully, so that the
+                                                             // reduction stack is indexed by constants
   const uint32_t W = (W_ > 0) ? (uint32_t)W_ : p.W;
 
   __shared__ uint64_t keys[kMaxWorkers];
@@ -193,103 +243,88 @@ __global__ void __launch_bounds__(256, MINB) la_sweep(const SweepParams p) {
     }
   }
 
+  // Grid-stride loop over coordinate groups, software-pipelined: while the replicas of one
+  // chunk are being consumed, the loads of the next chunk (or of the next group's first chunk
+  // and worker-independent data) are already in flight.  The empty asm statements pin that
+  // order against the compiler's scheduler.
   const uint64_t nthreads = (uint64_t)gridDim.x * blockDim.x;
-  for (uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < p.ngroups; grp += nthreads) {
+  uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (grp >= p.ngroups) return;
+  constexpr bool kLoadsBs = STEP && !PRE;
+
+  ReplicaChunk<CH> nxt;
+  CoordInputs in_next;
+  load_coord<GM, STEP, kLoadsBs>(in_next, p, grp * 4u);
+  load_chunk<CH>(nxt, p, W, 0u, grp * 4u);
+
+  for (;;) {
     const uint64_t off = grp * 4u;
-    GradInputs<GM> in;
-    if (STEP) {
-      if (GM == kGradQuadratic) {
-        in.a = ld_stream(p.a + off);
-        in.c = ld_stream(p.c + off);
-      }
-      if (GM == kGradNoiseScaled) in.s = ld_stream(p.s + off);
-      if (GM == kGradConstant) in.s = p.s ? ld_stream(p.s + off) : make_float4(1.f, 1.f, 1.f, 1.f);
-    }
+    const uint64_t next_grp = grp + nthreads;
+    const bool has_next = next_grp < p.ngroups;
+    const CoordInputs in = in_next;
     const uint64_t ctr0 = kGoldenGamma * (((p.j_base + off) >> 1) + 1u);
 
-    float4 bs;  // stale accumulator B^2_{t-t'}
-    if (!PRE && STEP) bs = ld_stream(p.Bs + off);
-
-    PairTree tree;
-    float4 xm, bm;
-    if (PRE) {
-      // ---- synchronisation of what is in memory: mean of x and B^2 over workers
-      for (uint32_t i0 = 0; i0 < W; i0 += CH) {
-        float4 xv[CH], bv[CH];
-#pragma unroll
-        for (int k = 0; k < CH; ++k)
-          if (i0 + k < W) {
-            xv[k] = ld_stream(p.X + (uint64_t)(i0 + k) * p.stride + off);
-            bv[k] = ld_stream(p.B2 + (uint64_t)(i0 + k) * p.stride + off);
-          }
-#pragma unroll
-        for (int k = 0; k < CH; ++k)
-          if (i0 + k < W) tree.push(i0 + k, xv[k], bv[k]);
-      }
-      tree.finish();
-      xm = div_by_workers<W_>(tree.x[0], W);
-      bm = div_by_workers<W_>(tree.b[0], W);
-      bs = bm;  // the mean accumulator is the new stale denominator
-      st_stream(p.Bs + off, bm);
-      if (!STEP) {
-        for (uint32_t i = 0; i < W; ++i) {
-          st_stream(p.X + (uint64_t)i * p.stride + off, xm);
-          st_stream(p.B2 + (uint64_t)i * p.stride + off, bm);
-        }
-        continue;
-      }
-    }
-
-    // ---- shared step size r = eta_t / sqrt(B^2_{t-t'} + t' eps^2), once per coordinate
     float4 r;
-    r.x = __fdiv_rn(eta_t, __fsqrt_rn(__fadd_rn(bs.x, q)));
-    r.y = __fdiv_rn(eta_t, __fsqrt_rn(__fadd_rn(bs.y, q)));
-    r.z = __fdiv_rn(eta_t, __fsqrt_rn(__fadd_rn(bs.z, q)));
-    r.w = __fdiv_rn(eta_t, __fsqrt_rn(__fadd_rn(bs.w, q)));
+    if (kLoadsBs) r = step_size(in.bs, q, eta_t);
+    PairTree tree;
 
-    if (PRE) {
-      // every replica starts the step from the mean
-      for (uint32_t i = 0; i < W; ++i) {
-        float4 xv = xm, bv = bm;
-        const float4 g = gradient4<GM, BF16>(p, in, xv, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
-        apply4(r, g, xv, bv);
-        st_stream(p.X + (uint64_t)i * p.stride + off, xv);
-        st_stream(p.B2 + (uint64_t)i * p.stride + off, bv);
+#pragma unroll kOuterUnroll
+    for (uint32_t i0 = 0; i0 < W; i0 += CH) {
+      ReplicaChunk<CH> cur = nxt;
+      if (i0 + CH < W) {
+        load_chunk<CH>(nxt, p, W, i0 + CH, off);
+      } else if (has_next) {
+        load_coord<GM, STEP, kLoadsBs>(in_next, p, next_grp * 4u);
+        load_chunk<CH>(nxt, p, W, 0u, next_grp * 4u);
       }
-    } else {
-      for (uint32_t i0 = 0; i0 < W; i0 += CH) {
-        float4 xv[CH], bv[CH];
+      asm volatile("" ::: "memory");
 #pragma unroll
-        for (int k = 0; k < CH; ++k)
-          if (i0 + k < W) {
-            xv[k] = ld_stream(p.X + (uint64_t)(i0 + k) * p.stride + off);
-            bv[k] = ld_stream(p.B2 + (uint64_t)(i0 + k) * p.stride + off);
-          }
-#pragma unroll
-        for (int k = 0; k < CH; ++k)
-          if (i0 + k < W) {
-            const uint32_t i = i0 + k;
-            const float4 g = gradient4<GM, BF16>(p, in, xv[k], kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
-            apply4(r, g, xv[k], bv[k]);
+      for (int k = 0; k < CH; ++k)
+        if (i0 + k < W) {
+          const uint32_t i = i0 + k;
+          if (PRE) {
+            tree.push(i, cur.x[k], cur.b[k]);
+          } else {
+            const float4 g = gradient4<GM, BF16>(p, in, cur.x[k], kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
+            apply4(r, g, cur.x[k], cur.b[k]);
             if (POST) {
-              tree.push(i, xv[k], bv[k]);
+              tree.push(i, cur.x[k], cur.b[k]);
             } else {
-              st_stream(p.X + (uint64_t)i * p.stride + off, xv[k]);
-              st_stream(p.B2 + (uint64_t)i * p.stride + off, bv[k]);
+              st_stream(p.X + (uint64_t)i * p.stride + off, cur.x[k]);
+              st_stream(p.B2 + (uint64_t)i * p.stride + off, cur.b[k]);
             }
           }
-      }
-      if (POST) {
-        tree.finish();
-        xm = div_by_workers<W_>(tree.x[0], W);
-        bm = div_by_workers<W_>(tree.b[0], W);
-        st_stream(p.Bs + off, bm);
+        }
+    }
+
+    if (PRE || POST) {
+      // synchronisation branch of Algorithm 3: means over workers; the mean accumulator is
+      // also the new stale denominator
+      tree.finish();
+      const float4 xm = div_by_workers<W_>(tree.x[0], W);
+      const float4 bm = div_by_workers<W_>(tree.b[0], W);
+      st_stream(p.Bs + off, bm);
+      if (PRE && STEP) {
+        // first step of the next period: every replica starts from the mean, t' = 1
+        r = step_size(bm, q, eta_t);
+#pragma unroll kOuterUnroll
+        for (uint32_t i = 0; i < W; ++i) {
+          float4 xv = xm, bv = bm;
+          const float4 g = gradient4<GM, BF16>(p, in, xv, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
+          apply4(r, g, xv, bv);
+          st_stream(p.X + (uint64_t)i * p.stride + off, xv);
+          st_stream(p.B2 + (uint64_t)i * p.stride + off, bv);
+        }
+      } else {
+#pragma unroll kOuterUnroll
         for (uint32_t i = 0; i < W; ++i) {
           st_stream(p.X + (uint64_t)i * p.stride + off, xm);
           st_stream(p.B2 + (uint64_t)i * p.stride + off, bm);
         }
       }
     }
+    if (!has_next) break;
+    grp = next_grp;
   }
 }
 
