@@ -320,6 +320,93 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+def run_report(args):
+    """All five configurations plus the synchronisation-period sweep of configuration 4
+    (H in {1,4,16,64} x {unfused, step+sync, sync+step}): per-kernel-class device time, GB/s
+    against the measured and the nominal HBM peak, share of time spent synchronising.
+    Writes one JSON document to --report-out and a markdown table to stdout."""
+    import torch
+    from paper_1911_09030_b200 import local_adaalter as la
+    from paper_1911_09030_b200 import workloads
+    torch.cuda.set_device(0)
+    peak, peak_kind = measured_peak()
+    rows = []
+
+    def one(wl, H, fusion, reps):
+        arr = wl.arrays()
+        ctx = la.LocalAdaAlter.with_torch_arena(wl.sizes, wl.W, wl.eta, wl.eps, H, b0sq=wl.b0sq)
+        if wl.grad == "quadratic":
+            ctx.set_grad_quadratic(wl.noise_seed, arr["a"], arr["c"], wl.sigma)
+        elif wl.grad == "noise_scaled":
+            ctx.set_grad_noise(wl.noise_seed, arr["s"])
+        else:
+            ctx.set_grad_noise(wl.noise_seed, None)
+        del arr
+        if wl.bf16_grads:
+            ctx.set_grad_dtype(la.LA_BF16)
+        ctx.set_fusion(fusion)
+        ctx.run(wl.T)                                   # warm-up: one full run
+        ctx.run(wl.T)
+        ctx.run(wl.T)
+        ctx.sync_stream()
+        ctx.get_stats(reset=True)
+        ctx.set_profiling(True)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        st = torch.cuda.current_stream()
+        e0.record(st)
+        for _ in range(reps):
+            ctx.run(wl.T)
+        e1.record(st)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        stats = ctx.get_stats(reset=True)
+        ctx.close()
+        row = {"config": wl.name, "W": wl.W, "N": wl.N, "H": H, "T": wl.T, "fusion": fusion,
+               "ms_per_run": ms, "updates_per_s": wl.W * wl.N * wl.T / (ms * 1e-3)}
+        tot_ms = sum(stats[f"ms_{c}"] for c in ("local", "sync", "fused"))
+        tot_b = sum(stats[f"bytes_{c}"] for c in ("local", "sync", "fused"))
+        row["GBps_all"] = tot_b / reps / (ms * 1e-3) / 1e9
+        for c in ("local", "sync", "fused"):
+            n = stats[f"launches_{c}"]
+            row[f"n_{c}"] = n // reps
+            row[f"us_{c}"] = 1e3 * stats[f"ms_{c}"] / n if n else None
+            row[f"GBps_{c}"] = stats[f"bytes_{c}"] / n / (stats[f"ms_{c}"] / n * 1e-3) / 1e9 if n else None
+            row[f"share_{c}"] = stats[f"ms_{c}"] / tot_ms if tot_ms else None
+        # time attributable to synchronising: stand-alone syncs, plus for fused passes the
+        # excess over a plain local step
+        us_local = row["us_local"] or row["us_fused"]
+        extra = 0.0
+        if row["n_sync"]:
+            extra += row["n_sync"] * row["us_sync"]
+        if row["n_fused"] and row["us_local"]:
+            extra += row["n_fused"] * max(0.0, row["us_fused"] - row["us_local"])
+        row["sync_share_of_time"] = extra / (1e3 * tot_ms / reps) if tot_ms else None
+        rows.append(row)
+        return row
+
+    for name in ("c1", "c2", "c3", "c5"):
+        wl = workloads.config(name)
+        one(wl, wl.H, args.fusion, reps=3 if name != "c1" else 20)
+    wl4 = workloads.config("c4")
+    for H in wl4.H_sweep:
+        for fusion in (0, 1, 2):
+            one(wl4, H, fusion, reps=2)
+    doc = {"peak_GBps": peak, "peak_kind": peak_kind, "nominal_GBps": NOMINAL_HBM_GBS, "rows": rows}
+    if args.report_out:
+        os.makedirs(os.path.dirname(os.path.abspath(args.report_out)), exist_ok=True)
+        with open(args.report_out, "w") as f:
+            json.dump(doc, f, indent=1)
+    f2 = lambda v, d=0: "-" if v is None else f"{v:.{d}f}"
+    print(f"| cfg | W | H | fusion | updates/s | GB/s all | pct of {peak:.0f} | pct of 8000 | K1 us (GB/s) | K2 us (GB/s) | "
+          "fused us (GB/s) | sync share |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|")
+    for r in rows:
+        print(f"| {r['config']} | {r['W']} | {r['H']} | {r['fusion']} | {r['updates_per_s']:.3e} | {r['GBps_all']:.0f} | "
+              f"{100 * r['GBps_all'] / peak:.1f} | {100 * r['GBps_all'] / NOMINAL_HBM_GBS:.1f} | "
+              f"{f2(r['us_local'], 1)} ({f2(r['GBps_local'])}) | {f2(r['us_sync'], 1)} ({f2(r['GBps_sync'])}) | "
+              f"{f2(r['us_fused'], 1)} ({f2(r['GBps_fused'])}) | {f2(100 * r['sync_share_of_time'], 1)} % |")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -332,9 +419,13 @@ def main():
     ap.add_argument("--fusion", type=int, default=1, help="0 unfused, 1 step+sync, 2 sync+next step")
     ap.add_argument("--blocks-per-sm", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--report", action="store_true", help="all configurations + the H sweep (not the JSON line)")
+    ap.add_argument("--report-out", default=None)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
+    if args.report:
+        return run_report(args)
     from paper_1911_09030_b200 import workloads
     wl = workloads.config(args.workload)
     if args.H is not None:
