@@ -115,7 +115,7 @@ int la_set_warmup(la_ctx* ctx, uint32_t warm_up_steps);
 int la_set_fusion(la_ctx* ctx, int mode);
 /* Tuning knob: the sweep kernels run as a grid-stride loop over at most
  * blocks_per_sm * (number of SMs) blocks of 256 threads; 0 restores the built-in
- * per-kernel defaults (48 for kernels that take a step, unbounded for the pure sync). */
+ * per-kernel defaults (96 for kernels that take a step, unbounded for the pure sync). */
 int la_set_launch_shape(la_ctx* ctx, int blocks_per_sm);
 /* Record CUDA events around every launch and accumulate device time per class. */
 int la_set_profiling(la_ctx* ctx, int on);

@@ -16,14 +16,14 @@
 
 namespace la {
 
-SweepFn lookup_sweep_w0(int, bool, bool, bool, bool);
-SweepFn lookup_sweep_w1(int, bool, bool, bool, bool);
-SweepFn lookup_sweep_w2(int, bool, bool, bool, bool);
-SweepFn lookup_sweep_w4(int, bool, bool, bool, bool);
-SweepFn lookup_sweep_w8(int, bool, bool, bool, bool);
-SweepFn lookup_sweep_w16(int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w0(int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w1(int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w2(int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w4(int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w8(int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w16(int, bool, bool, bool, bool);
 
-SweepFn lookup_sweep(int W, int gm, bool bf16, bool pre, bool step, bool post) {
+SweepKernel lookup_sweep(int W, int gm, bool bf16, bool pre, bool step, bool post) {
   switch (W) {
     case 1: return lookup_sweep_w1(gm, bf16, pre, step, post);
     case 2: return lookup_sweep_w2(gm, bf16, pre, step, post);
@@ -206,23 +206,25 @@ double pass_bytes(const la_ctx* c, bool pre, bool step, bool post, int gm) {
 }
 
 int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t tp, int gm, const void* gext) {
-  la::SweepFn fn = la::lookup_sweep((int)c->W, gm, c->bf16 && gm <= la::kGradQuadratic, pre, step, post);
+  const la::SweepKernel k = la::lookup_sweep((int)c->W, gm, c->bf16 && gm <= la::kGradQuadratic, pre, step, post);
+  la::SweepFn fn = k.fn;
   if (!fn) return fail(c, LA_ESTATE, "no kernel for this combination (W=%u grad=%d)", c->W, gm);
   la::SweepParams p{};
   p.X = c->X; p.B2 = c->B2; p.Bs = c->Bs;
   p.a = c->pa; p.c = c->pc; p.s = c->has_s ? c->ps : nullptr;
   p.gext = gext;
-  p.n = c->N; p.ngroups = c->ngroups; p.stride = c->stride; p.j_base = c->j_base;
+  p.n = c->N; p.stride = c->stride; p.j_base = c->j_base;
   p.seed = c->seed; p.t = t; p.W = c->W; p.tp = tp;
   p.warm_up_steps = c->warm_up_steps; p.identical_workers = c->identical ? 1u : 0u;
   p.eta = c->eta; p.eps = c->eps; p.sigma = c->sigma;
   const unsigned block = la::kBlockThreads;
-  uint64_t blocks = (c->ngroups + block - 1) / block;
-  // Measured on B200: kernels that generate gradients run best with about 48 blocks per SM in
-  // the grid (each thread then handles a few coordinate groups, so the software pipeline pays
-  // off, while blocks are still small enough to balance the SMs); the pure averaging kernel
-  // runs best with one group per thread.
-  const int bps = c->blocks_per_sm > 0 ? c->blocks_per_sm : (step ? 48 : 4096);
+  const uint64_t ngroups = (c->N + (uint64_t)k.vec - 1) / (uint64_t)k.vec;
+  uint64_t blocks = (ngroups + block - 1) / block;
+  // Measured on B200 (sweep of 6..4096 blocks per SM): kernels that take a step run best when a
+  // thread handles a few coordinate groups (96 blocks per SM in the grid: the software pipeline
+  // pays off while blocks stay small enough to balance the SMs); the pure averaging kernel runs
+  // best with one group per thread.
+  const int bps = c->blocks_per_sm > 0 ? c->blocks_per_sm : (step ? 96 : 4096);
   const uint64_t cap = (uint64_t)c->num_sms * (uint64_t)bps;
   if (blocks > cap) blocks = cap;
   const int cls = (step && (pre || post)) ? kClassFused : (step ? kClassLocal : kClassSync);

@@ -41,8 +41,7 @@ struct SweepParams {
   const float* s;  // [stride] or null
   const void* gext;    // external gradients, [W][N]
   uint64_t n;          // logical coordinates N
-  uint64_t ngroups;    // ceil(N / 4)
-  uint64_t stride;     // replica stride in floats (multiple of 64, >= 4*ngroups)
+  uint64_t stride;     // replica stride in floats (multiple of 64, >= N rounded up to 4)
   uint64_t j_base;     // global index of coordinate 0 (multiple of 4)
   uint64_t seed;
   uint64_t t;          // 1-based global step index of the STEP part
@@ -56,158 +55,6 @@ struct SweepParams {
 constexpr int kMaxWorkers = 64;
 constexpr int kTreeDepth = 7;  // log2(kMaxWorkers) + 1 partial sums
 
-__device__ __forceinline__ float4 ld_stream(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
-__device__ __forceinline__ void st_stream(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
-
-__device__ __forceinline__ float4 add4(float4 l, float4 r) {
-  return make_float4(__fadd_rn(l.x, r.x), __fadd_rn(l.y, r.y), __fadd_rn(l.z, r.z), __fadd_rn(l.w, r.w));
-}
-
-// Mean over workers = adjacent-pair tree sum, then one division by (float)W.  For a power of
-// two the division is replaced by the multiplication with the exact reciprocal, which rounds
-// the same real number and therefore gives the same bits.
-template <int W_>
-__device__ __forceinline__ float4 div_by_workers(float4 v, uint32_t W) {
-  if (W_ > 0 && (W_ & (W_ - 1)) == 0) {
-    const float inv = 1.0f / (float)W_;
-    return make_float4(__fmul_rn(v.x, inv), __fmul_rn(v.y, inv), __fmul_rn(v.z, inv), __fmul_rn(v.w, inv));
-  }
-  const float w = __uint2float_rn(W);
-  return make_float4(__fdiv_rn(v.x, w), __fdiv_rn(v.y, w), __fdiv_rn(v.z, w), __fdiv_rn(v.w, w));
-}
-
-// Streaming form of the adjacent-pair tree: a stack of partial sums, one per level, merged
-// like the carries of a binary counter.  After pushing worker i the two top entries are
-// merged once for every trailing zero bit of (i+1); left operand = older entry.  With W known
-// at compile time the loop unrolls and every stack index is a constant (registers only).
-struct PairTree {
-  float4 x[kTreeDepth], b[kTreeDepth];
-  int sp = 0;
-  __device__ __forceinline__ void push(uint32_t i, float4 vx, float4 vb) {
-    x[sp] = vx;
-    b[sp] = vb;
-    ++sp;
-    for (uint32_t cnt = i + 1u; (cnt & 1u) == 0u; cnt >>= 1) {
-      --sp;
-      x[sp - 1] = add4(x[sp - 1], x[sp]);
-      b[sp - 1] = add4(b[sp - 1], b[sp]);
-    }
-  }
-  __device__ __forceinline__ void finish() {
-    while (sp > 1) {
-      --sp;
-      x[sp - 1] = add4(x[sp - 1], x[sp]);
-      b[sp - 1] = add4(b[sp - 1], b[sp]);
-    }
-  }
-};
-
-// Worker-independent data of one coordinate group: the stale accumulator and the problem arrays.
-struct CoordInputs {
-  float4 bs, a, c, s;
-};
-
-template <int GM, bool STEP, bool LOAD_BS>
-__device__ __forceinline__ void load_coord(CoordInputs& in, const SweepParams& p, uint64_t off) {
-  if (LOAD_BS) in.bs = ld_stream(p.Bs + off);
-  if (STEP) {
-    if (GM == kGradQuadratic) {
-      in.a = ld_stream(p.a + off);
-      in.c = ld_stream(p.c + off);
-    }
-    if (GM == kGradNoiseScaled) in.s = ld_stream(p.s + off);
-    if (GM == kGradConstant) in.s = p.s ? ld_stream(p.s + off) : make_float4(1.f, 1.f, 1.f, 1.f);
-  }
-}
-
-// x and B^2 of CH consecutive replicas for one coordinate group.
-template <int CH>
-struct ReplicaChunk {
-  float4 x[CH], b[CH];
-};
-
-template <int CH>
-__device__ __forceinline__ void load_chunk(ReplicaChunk<CH>& ch, const SweepParams& p, uint32_t W, uint32_t i0,
-                                           uint64_t off) {
-#pragma unroll
-  for (int k = 0; k < CH; ++k)
-    if (i0 + k < W) {
-      ch.x[k] = ld_stream(p.X + (uint64_t)(i0 + k) * p.stride + off);
-      ch.b[k] = ld_stream(p.B2 + (uint64_t)(i0 + k) * p.stride + off);
-    }
-}
-
-// r = eta_t / sqrt(B^2_{t-t'} + t' eps^2): the step size all workers share (Section 4.2).
-__device__ __forceinline__ float4 step_size(float4 bs, float q, float eta_t) {
-  float4 r;
-  r.x = __fdiv_rn(eta_t, __fsqrt_rn(__fadd_rn(bs.x, q)));
-  r.y = __fdiv_rn(eta_t, __fsqrt_rn(__fadd_rn(bs.y, q)));
-  r.z = __fdiv_rn(eta_t, __fsqrt_rn(__fadd_rn(bs.z, q)));
-  r.w = __fdiv_rn(eta_t, __fsqrt_rn(__fadd_rn(bs.w, q)));
-  return r;
-}
-
-// Gradient of four coordinates for one worker.  `xv` is the worker's own iterate
-// (Algorithm 3: G_{i,t} = grad f(x_{i,t-1}; z_{i,t})).
-template <int GM, bool BF16>
-__device__ __forceinline__ float4 gradient4(const SweepParams& p, const CoordInputs& in, float4 xv,
-                                            uint64_t key, uint64_t ctr0, uint32_t worker, uint64_t off) {
-  float4 g;
-  if (GM == kGradConstant) {
-    return in.s;
-  } else if (GM == kGradExternalF32 || GM == kGradExternalBF16) {
-    const uint64_t base = (uint64_t)worker * p.n + off;
-    float v[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      v[k] = 0.0f;
-      if (off + k < p.n) {
-        if (GM == kGradExternalF32) {
-          v[k] = __ldcs(reinterpret_cast<const float*>(p.gext) + base + k);
-        } else {
-          const unsigned short h = __ldcs(reinterpret_cast<const unsigned short*>(p.gext) + base + k);
-          v[k] = __uint_as_float((uint32_t)h << 16);
-        }
-      }
-    }
-    return make_float4(v[0], v[1], v[2], v[3]);
-  } else {
-    float4 xi;
-    normal_pair(key, ctr0, xi.x, xi.y);
-    normal_pair(key, ctr0 + kGoldenGamma, xi.z, xi.w);
-    if (GM == kGradNoise) {
-      g = xi;
-    } else if (GM == kGradNoiseScaled) {
-      g = make_float4(__fmul_rn(in.s.x, xi.x), __fmul_rn(in.s.y, xi.y), __fmul_rn(in.s.z, xi.z),
-                      __fmul_rn(in.s.w, xi.w));
-    } else {  // quadratic
-      g.x = __fmaf_rn(in.a.x, __fsub_rn(xv.x, in.c.x), __fmul_rn(p.sigma, xi.x));
-      g.y = __fmaf_rn(in.a.y, __fsub_rn(xv.y, in.c.y), __fmul_rn(p.sigma, xi.y));
-      g.z = __fmaf_rn(in.a.z, __fsub_rn(xv.z, in.c.z), __fmul_rn(p.sigma, xi.z));
-      g.w = __fmaf_rn(in.a.w, __fsub_rn(xv.w, in.c.w), __fmul_rn(p.sigma, xi.w));
-    }
-    if (BF16) {
-      g.x = round_through_bf16(g.x);
-      g.y = round_through_bf16(g.y);
-      g.z = round_through_bf16(g.z);
-      g.w = round_through_bf16(g.w);
-    }
-  }
-  return g;
-}
-
-// y = x - r g ; A^2 = B^2 + g g   (Algorithm 3), one fused multiply-add each.
-__device__ __forceinline__ void apply4(float4 r, float4 g, float4& x, float4& b) {
-  x.x = __fmaf_rn(-r.x, g.x, x.x);
-  x.y = __fmaf_rn(-r.y, g.y, x.y);
-  x.z = __fmaf_rn(-r.z, g.z, x.z);
-  x.w = __fmaf_rn(-r.w, g.w, x.w);
-  b.x = __fmaf_rn(g.x, g.x, b.x);
-  b.y = __fmaf_rn(g.y, g.y, b.y);
-  b.z = __fmaf_rn(g.z, g.z, b.z);
-  b.w = __fmaf_rn(g.w, g.w, b.w);
-}
-
 #ifndef LA_BLOCK
 #define LA_BLOCK 256
 #endif
@@ -216,9 +63,220 @@ __device__ __forceinline__ void apply4(float4 r, float4 g, float4& x, float4& b)
 #endif
 constexpr int kBlockThreads = LA_BLOCK;
 
-template <int W_, int GM, bool BF16, bool PRE, bool STEP, bool POST, int MINB>
+// V consecutive coordinates held by one thread (V = 4: one 128-bit access, two Box-Muller
+// pairs; V = 2: one 64-bit access, one pair).
+template <int V>
+struct Vec {
+  float v[V];
+};
+
+// Row addresses are carried as running 64-bit byte addresses that advance by one replica stride
+// per worker.  The advance is an opaque add so that the compiler keeps ONE running pointer
+// instead of hoisting a separate loop-invariant row base per worker out of the grid-stride loop
+// (2W 64-bit bases = up to 64 registers, which would halve the occupancy).
+__device__ __forceinline__ void advance(uint64_t& addr, uint64_t bytes) {
+  asm volatile("add.u64 %0, %0, %1;" : "+l"(addr) : "l"(bytes));
+}
+__device__ __forceinline__ const float* as_ptr(uint64_t addr) { return reinterpret_cast<const float*>(addr); }
+__device__ __forceinline__ float* as_mut(uint64_t addr) { return reinterpret_cast<float*>(addr); }
+
+template <int V>
+__device__ __forceinline__ Vec<V> ld_stream(const float* p) {
+  Vec<V> r;
+  if (V == 4) {
+    const float4 t = __ldcs(reinterpret_cast<const float4*>(p));
+    r.v[0] = t.x; r.v[1] = t.y; r.v[V - 2] = t.z; r.v[V - 1] = t.w;
+  } else {
+    const float2 t = __ldcs(reinterpret_cast<const float2*>(p));
+    r.v[0] = t.x; r.v[1] = t.y;
+  }
+  return r;
+}
+
+template <int V>
+__device__ __forceinline__ void st_stream(float* p, const Vec<V>& a) {
+  if (V == 4) {
+    __stcs(reinterpret_cast<float4*>(p), make_float4(a.v[0], a.v[1], a.v[V - 2], a.v[V - 1]));
+  } else {
+    __stcs(reinterpret_cast<float2*>(p), make_float2(a.v[0], a.v[1]));
+  }
+}
+
+template <int V>
+__device__ __forceinline__ Vec<V> splat(float f) {
+  Vec<V> r;
+#pragma unroll
+  for (int k = 0; k < V; ++k) r.v[k] = f;
+  return r;
+}
+
+template <int V>
+__device__ __forceinline__ Vec<V> add(const Vec<V>& l, const Vec<V>& r) {
+  Vec<V> o;
+#pragma unroll
+  for (int k = 0; k < V; ++k) o.v[k] = __fadd_rn(l.v[k], r.v[k]);
+  return o;
+}
+
+// Mean over workers = adjacent-pair tree sum, then one division by (float)W.  For a power of
+// two the division is replaced by the multiplication with the exact reciprocal, which rounds
+// the same real number and therefore gives the same bits.
+template <int W_, int V>
+__device__ __forceinline__ Vec<V> div_by_workers(const Vec<V>& a, uint32_t W) {
+  Vec<V> o;
+  if (W_ > 0 && (W_ & (W_ - 1)) == 0) {
+    const float inv = 1.0f / (float)W_;
+#pragma unroll
+    for (int k = 0; k < V; ++k) o.v[k] = __fmul_rn(a.v[k], inv);
+  } else {
+    const float w = __uint2float_rn(W);
+#pragma unroll
+    for (int k = 0; k < V; ++k) o.v[k] = __fdiv_rn(a.v[k], w);
+  }
+  return o;
+}
+
+// Streaming form of the adjacent-pair tree: a stack of partial sums, one per level, merged
+// like the carries of a binary counter.  After pushing worker i the two top entries are
+// merged once for every trailing zero bit of (i+1); left operand = older entry.  With W known
+// at compile time the loop unrolls and every stack index is a constant (registers only).
+template <int V>
+struct PairTree {
+  Vec<V> x[kTreeDepth], b[kTreeDepth];
+  int sp = 0;
+  __device__ __forceinline__ void push(uint32_t i, const Vec<V>& vx, const Vec<V>& vb) {
+    x[sp] = vx;
+    b[sp] = vb;
+    ++sp;
+    for (uint32_t cnt = i + 1u; (cnt & 1u) == 0u; cnt >>= 1) {
+      --sp;
+      x[sp - 1] = add(x[sp - 1], x[sp]);
+      b[sp - 1] = add(b[sp - 1], b[sp]);
+    }
+  }
+  __device__ __forceinline__ void finish() {
+    while (sp > 1) {
+      --sp;
+      x[sp - 1] = add(x[sp - 1], x[sp]);
+      b[sp - 1] = add(b[sp - 1], b[sp]);
+    }
+  }
+};
+
+// Worker-independent data of one coordinate group: the stale accumulator and the problem arrays.
+template <int V>
+struct CoordInputs {
+  Vec<V> bs, a, c, s;
+};
+
+template <int GM, bool STEP, bool LOAD_BS, int V>
+__device__ __forceinline__ void load_coord(CoordInputs<V>& in, const SweepParams& p, uint64_t off) {
+  if (LOAD_BS) in.bs = ld_stream<V>(p.Bs + off);
+  if (STEP) {
+    if (GM == kGradQuadratic) {
+      in.a = ld_stream<V>(p.a + off);
+      in.c = ld_stream<V>(p.c + off);
+    }
+    if (GM == kGradNoiseScaled) in.s = ld_stream<V>(p.s + off);
+    if (GM == kGradConstant) in.s = p.s ? ld_stream<V>(p.s + off) : splat<V>(1.0f);
+  }
+}
+
+// x and B^2 of CH consecutive replicas for one coordinate group.
+template <int V, int CH>
+struct ReplicaChunk {
+  Vec<V> x[CH], b[CH];
+};
+
+// Loads replicas i0 .. i0+CH-1; `addr` is the address of x of replica i0 for this coordinate
+// group and is left pointing at replica i0+CH.  B^2 of a replica sits `b_delta` bytes after x.
+template <int V, int CH>
+__device__ __forceinline__ void load_chunk(ReplicaChunk<V, CH>& ch, uint64_t& addr, uint64_t b_delta,
+                                           uint64_t stride_bytes, uint32_t W, uint32_t i0) {
+#pragma unroll
+  for (int k = 0; k < CH; ++k)
+    if (i0 + k < W) {
+      ch.x[k] = ld_stream<V>(as_ptr(addr));
+      ch.b[k] = ld_stream<V>(as_ptr(addr + b_delta));
+      advance(addr, stride_bytes);
+    }
+}
+
+// Stores x and B^2 of one replica at `addr` and advances to the next replica.
+template <int V>
+__device__ __forceinline__ void store_replica(uint64_t& addr, uint64_t b_delta, uint64_t stride_bytes,
+                                              const Vec<V>& x, const Vec<V>& b) {
+  st_stream<V>(as_mut(addr), x);
+  st_stream<V>(as_mut(addr + b_delta), b);
+  advance(addr, stride_bytes);
+}
+
+// r = eta_t / sqrt(B^2_{t-t'} + t' eps^2): the step size all workers share (Section 4.2).
+template <int V>
+__device__ __forceinline__ Vec<V> step_size(const Vec<V>& bs, float q, float eta_t) {
+  Vec<V> r;
+#pragma unroll
+  for (int k = 0; k < V; ++k) r.v[k] = __fdiv_rn(eta_t, __fsqrt_rn(__fadd_rn(bs.v[k], q)));
+  return r;
+}
+
+// Gradient of V coordinates for one worker.  `xv` is the worker's own iterate
+// (Algorithm 3: G_{i,t} = grad f(x_{i,t-1}; z_{i,t})).  `ctr0` = gamma (p0 + 1) for the
+// group's first coordinate pair p0.
+template <int GM, bool BF16, int V>
+__device__ __forceinline__ Vec<V> gradient(const SweepParams& p, const CoordInputs<V>& in, const Vec<V>& xv,
+                                           uint64_t key, uint64_t ctr0, uint32_t worker, uint64_t off) {
+  Vec<V> g;
+  if (GM == kGradConstant) {
+    return in.s;
+  } else if (GM == kGradExternalF32 || GM == kGradExternalBF16) {
+    const uint64_t base = (uint64_t)worker * p.n + off;
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+      g.v[k] = 0.0f;
+      if (off + k < p.n) {
+        if (GM == kGradExternalF32) {
+          g.v[k] = __ldcs(reinterpret_cast<const float*>(p.gext) + base + k);
+        } else {
+          const unsigned short h = __ldcs(reinterpret_cast<const unsigned short*>(p.gext) + base + k);
+          g.v[k] = __uint_as_float((uint32_t)h << 16);  // bf16 -> fp32 is exact
+        }
+      }
+    }
+    return g;
+  } else {
+    Vec<V> xi;
+#pragma unroll
+    for (int k = 0; k < V; k += 2) normal_pair(key, ctr0 + kGoldenGamma * (uint64_t)(k / 2), xi.v[k], xi.v[k + 1]);
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+      if (GM == kGradNoise) {
+        g.v[k] = xi.v[k];
+      } else if (GM == kGradNoiseScaled) {
+        g.v[k] = __fmul_rn(in.s.v[k], xi.v[k]);
+      } else {  // quadratic
+        g.v[k] = __fmaf_rn(in.a.v[k], __fsub_rn(xv.v[k], in.c.v[k]), __fmul_rn(p.sigma, xi.v[k]));
+      }
+      if (BF16) g.v[k] = round_through_bf16(g.v[k]);
+    }
+  }
+  return g;
+}
+
+// y = x - r g ; A^2 = B^2 + g g   (Algorithm 3), one fused multiply-add each.
+template <int V>
+__device__ __forceinline__ void apply(const Vec<V>& r, const Vec<V>& g, Vec<V>& x, Vec<V>& b) {
+#pragma unroll
+  for (int k = 0; k < V; ++k) {
+    x.v[k] = __fmaf_rn(-r.v[k], g.v[k], x.v[k]);
+    b.v[k] = __fmaf_rn(g.v[k], g.v[k], b.v[k]);
+  }
+}
+
+template <int W_, int V, int GM, bool BF16, bool PRE, bool STEP, bool POST, int MINB>
 __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) {
   static_assert(!(PRE && POST), "one synchronisation per pass");
+  static_assert(V == 2 || V == 4, "a thread owns 2 or 4 coordinates");
   constexpr bool kNeedsNoise = STEP && (GM == kGradNoise || GM == kGradNoiseScaled || GM == kGradQuadratic);
   constexpr int CH = (W_ > 0) ? (W_ < LA_CH ? W_ : LA_CH) : 4;  // replicas loaded before any is consumed
   constexpr int kOuterUnroll = (W_ > 0) ? kMaxWorkers : 1;  // static W: unroll fully, so that the
@@ -247,35 +305,43 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
   // chunk are being consumed, the loads of the next chunk (or of the next group's first chunk
   // and worker-independent data) are already in flight.  The empty asm statements pin that
   // order against the compiler's scheduler.
+  const uint64_t ngroups = (p.n + (uint64_t)(V - 1)) / (uint64_t)V;
   const uint64_t nthreads = (uint64_t)gridDim.x * blockDim.x;
   uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (grp >= p.ngroups) return;
+  if (grp >= ngroups) return;
   constexpr bool kLoadsBs = STEP && !PRE;
 
-  ReplicaChunk<CH> nxt;
-  CoordInputs in_next;
-  load_coord<GM, STEP, kLoadsBs>(in_next, p, grp * 4u);
-  load_chunk<CH>(nxt, p, W, 0u, grp * 4u);
+  const uint64_t x_base = reinterpret_cast<uint64_t>(p.X);
+  const uint64_t b_delta = reinterpret_cast<uint64_t>(p.B2) - x_base;
+  const uint64_t stride_bytes = p.stride * sizeof(float);
+
+  ReplicaChunk<V, CH> nxt;
+  CoordInputs<V> in_next;
+  load_coord<GM, STEP, kLoadsBs, V>(in_next, p, grp * V);
+  uint64_t ld_addr = x_base + grp * (V * sizeof(float));
+  load_chunk<V, CH>(nxt, ld_addr, b_delta, stride_bytes, W, 0u);
 
   for (;;) {
-    const uint64_t off = grp * 4u;
+    const uint64_t off = grp * V;
     const uint64_t next_grp = grp + nthreads;
-    const bool has_next = next_grp < p.ngroups;
-    const CoordInputs in = in_next;
+    const bool has_next = next_grp < ngroups;
+    const CoordInputs<V> in = in_next;
     const uint64_t ctr0 = kGoldenGamma * (((p.j_base + off) >> 1) + 1u);
+    uint64_t st_addr = x_base + off * sizeof(float);
 
-    float4 r;
-    if (kLoadsBs) r = step_size(in.bs, q, eta_t);
-    PairTree tree;
+    Vec<V> r;
+    if (kLoadsBs) r = step_size<V>(in.bs, q, eta_t);
+    PairTree<V> tree;
 
 #pragma unroll kOuterUnroll
     for (uint32_t i0 = 0; i0 < W; i0 += CH) {
-      ReplicaChunk<CH> cur = nxt;
+      ReplicaChunk<V, CH> cur = nxt;
       if (i0 + CH < W) {
-        load_chunk<CH>(nxt, p, W, i0 + CH, off);
+        load_chunk<V, CH>(nxt, ld_addr, b_delta, stride_bytes, W, i0 + CH);
       } else if (has_next) {
-        load_coord<GM, STEP, kLoadsBs>(in_next, p, next_grp * 4u);
-        load_chunk<CH>(nxt, p, W, 0u, next_grp * 4u);
+        load_coord<GM, STEP, kLoadsBs, V>(in_next, p, next_grp * V);
+        ld_addr = x_base + next_grp * (V * sizeof(float));
+        load_chunk<V, CH>(nxt, ld_addr, b_delta, stride_bytes, W, 0u);
       }
       asm volatile("" ::: "memory");
 #pragma unroll
@@ -285,13 +351,12 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
           if (PRE) {
             tree.push(i, cur.x[k], cur.b[k]);
           } else {
-            const float4 g = gradient4<GM, BF16>(p, in, cur.x[k], kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
-            apply4(r, g, cur.x[k], cur.b[k]);
+            const Vec<V> g = gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
+            apply<V>(r, g, cur.x[k], cur.b[k]);
             if (POST) {
               tree.push(i, cur.x[k], cur.b[k]);
             } else {
-              st_stream(p.X + (uint64_t)i * p.stride + off, cur.x[k]);
-              st_stream(p.B2 + (uint64_t)i * p.stride + off, cur.b[k]);
+              store_replica<V>(st_addr, b_delta, stride_bytes, cur.x[k], cur.b[k]);
             }
           }
         }
@@ -301,26 +366,22 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
       // synchronisation branch of Algorithm 3: means over workers; the mean accumulator is
       // also the new stale denominator
       tree.finish();
-      const float4 xm = div_by_workers<W_>(tree.x[0], W);
-      const float4 bm = div_by_workers<W_>(tree.b[0], W);
-      st_stream(p.Bs + off, bm);
+      const Vec<V> xm = div_by_workers<W_, V>(tree.x[0], W);
+      const Vec<V> bm = div_by_workers<W_, V>(tree.b[0], W);
+      st_stream<V>(p.Bs + off, bm);
       if (PRE && STEP) {
         // first step of the next period: every replica starts from the mean, t' = 1
-        r = step_size(bm, q, eta_t);
+        r = step_size<V>(bm, q, eta_t);
 #pragma unroll kOuterUnroll
         for (uint32_t i = 0; i < W; ++i) {
-          float4 xv = xm, bv = bm;
-          const float4 g = gradient4<GM, BF16>(p, in, xv, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
-          apply4(r, g, xv, bv);
-          st_stream(p.X + (uint64_t)i * p.stride + off, xv);
-          st_stream(p.B2 + (uint64_t)i * p.stride + off, bv);
+          Vec<V> xv = xm, bv = bm;
+          const Vec<V> g = gradient<GM, BF16, V>(p, in, xv, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
+          apply<V>(r, g, xv, bv);
+          store_replica<V>(st_addr, b_delta, stride_bytes, xv, bv);
         }
       } else {
 #pragma unroll kOuterUnroll
-        for (uint32_t i = 0; i < W; ++i) {
-          st_stream(p.X + (uint64_t)i * p.stride + off, xm);
-          st_stream(p.B2 + (uint64_t)i * p.stride + off, bm);
-        }
+        for (uint32_t i = 0; i < W; ++i) store_replica<V>(st_addr, b_delta, stride_bytes, xm, bm);
       }
     }
     if (!has_next) break;
@@ -328,8 +389,12 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
   }
 }
 
-// Host-side launcher table entry.
+// Host-side launcher table entry: the kernel and the number of coordinates a thread owns.
 using SweepFn = void (*)(const SweepParams);
-SweepFn lookup_sweep(int W, int gm, bool bf16, bool pre, bool step, bool post);
+struct SweepKernel {
+  SweepFn fn;
+  int vec;
+};
+SweepKernel lookup_sweep(int W, int gm, bool bf16, bool pre, bool step, bool post);
 
 }  // namespace la
