@@ -194,7 +194,8 @@ def run_ours(args, wl):
         torch.cuda.synchronize()
 
     # this rank's coordinate range: the same configuration, shifted (weak scaling)
-    j_base = rank * ((wl.N + 3) // 4 * 4)
+    from paper_1911_09030_b200 import sharding
+    j_base = sharding.weak_scaling_base(wl.N, rank)
     arr = wl.arrays()            # same per-coordinate inputs on every rank; noise differs through j_base
     stream = torch.cuda.current_stream()
     ctx = la.LocalAdaAlter.with_torch_arena(wl.sizes, wl.W, wl.eta, wl.eps, wl.H, b0sq=wl.b0sq, j_base=j_base)
@@ -262,10 +263,8 @@ def run_ours(args, wl):
     barrier()
     e2e_ms = 1e3 * (time.perf_counter() - t0) / e2e_steps
 
-    t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = float(t[0]), float(t[1])
+    ms_total = sharding.max_over_ranks(ms_total, dist if world > 1 else None)
+    e2e_ms = sharding.max_over_ranks(e2e_ms, dist if world > 1 else None)
     ms_per_step = ms_total / args.steps
     units = wl.W * wl.N * wl.T * world
     value = units / (ms_per_step * 1e-3)
