@@ -17,6 +17,7 @@
 //     synchronisation and is the same on every worker          Section 4.2,
 //     "Lazy update of the denominators"; Appendix A (definition of B-bar)
 //   * warm-up eta_t = eta*min(1, t/warm_up_steps)               Section 6.2
+//   * baselines: Distributed AdaGrad (Algorithm 1), Local SGD (Algorithm 2)
 //
 // Two state copies advance side by side:
 //   fp32 : the arithmetic contract (one IEEE-754 binary32 operation per line
@@ -176,6 +177,7 @@ T tree_sum(std::vector<T>& v) {
 }
 
 enum GradMode { kNoise = 0, kQuadratic = 1, kConstant = 2 };
+enum Rule { kRuleAdaAlter = 0, kRuleLocalSGD = 1, kRuleAdaGrad = 2 };
 
 struct Oracle {
   uint64_t n = 0;        // coordinates simulated here
@@ -183,6 +185,7 @@ struct Oracle {
   uint32_t W = 0, H = 0;
   float eta = 0, eps = 0, b0sq = 0;
   uint32_t warm_up_steps = 0;  // 0 = no warm-up
+  int rule = kRuleAdaAlter;    // Algorithm 3 by default; Algorithms 1 and 2 as baselines
   // gradient source
   int mode = kNoise;
   uint64_t seed = 0;
@@ -209,18 +212,54 @@ struct Oracle {
     return (double)eta * std::fmin(1.0, ratio);
   }
 
+  // Stochastic gradient G_{i,t} of worker i at coordinate j, evaluated at the iterate stored at
+  // index ix (fp32: g from X[ix]; shadow: gd from Xd[ix]).  `gext` prescribes it instead.
+  void gradient(uint32_t i, uint64_t j, size_t ix, uint64_t key_i, const float* gext, float* g_out,
+                double* gd_out) const {
+    float g;
+    double gd;
+    if (gext) {
+      g = gext[(size_t)i * n + j];
+      gd = (double)g;
+    } else if (mode == kConstant) {
+      g = s.empty() ? 1.0f : s[j];
+      gd = (double)g;
+    } else {
+      float xi = noise_xi(key_i, j_base + j);
+      if (mode == kNoise) {
+        g = s.empty() ? xi : s[j] * xi;
+        gd = s.empty() ? (double)xi : (double)s[j] * (double)xi;
+      } else {
+        float dlt = X[ix] - c[j];
+        float nz = sigma * xi;
+        g = std::fmaf(a[j], dlt, nz);
+        gd = (double)a[j] * (Xd[ix] - (double)c[j]) + (double)sigma * (double)xi;
+      }
+      if (bf16) {
+        g = bf16_round(g);
+        gd = (double)bf16_round((float)gd);
+      }
+    }
+    *g_out = g;
+    *gd_out = gd;
+  }
+
+  std::vector<uint64_t> step_keys() const {
+    std::vector<uint64_t> key(W);
+    for (uint32_t i = 0; i < W; ++i) key[i] = stream_key(seed, t, identical_workers ? 0u : i);
+    return key;
+  }
+
   // One iteration of Algorithm 3 without the synchronisation branch.
   // `gext` (optional) supplies G_{i,t} as a [W][n] table instead of the source.
-  void local_step(const float* gext) {
+  void adaalter_step(const float* gext) {
     t += 1;
     tp += 1;
     const float eps2 = eps * eps;
     const float et = eta_t();
     const double etd = eta_t_d();
     const double eps2d = (double)eps * (double)eps;
-    std::vector<uint64_t> key(W);
-    for (uint32_t i = 0; i < W; ++i)
-      key[i] = stream_key(seed, t, identical_workers ? 0u : i);
+    const std::vector<uint64_t> key = step_keys();
     for (uint64_t j = 0; j < n; ++j) {
       // shared, stale denominator: B^2 as of the last sync + t' eps^2
       float q = (float)tp * eps2;
@@ -231,28 +270,7 @@ struct Oracle {
         size_t ix = (size_t)i * n + j;
         float g;
         double gd;
-        if (gext) {
-          g = gext[ix];
-          gd = (double)g;
-        } else if (mode == kConstant) {
-          g = s.empty() ? 1.0f : s[j];
-          gd = (double)g;
-        } else {
-          float xi = noise_xi(key[i], j_base + j);
-          if (mode == kNoise) {
-            g = s.empty() ? xi : s[j] * xi;
-            gd = s.empty() ? (double)xi : (double)s[j] * (double)xi;
-          } else {
-            float dlt = X[ix] - c[j];
-            float nz = sigma * xi;
-            g = std::fmaf(a[j], dlt, nz);
-            gd = (double)a[j] * (Xd[ix] - (double)c[j]) + (double)sigma * (double)xi;
-          }
-          if (bf16) {
-            g = bf16_round(g);
-            gd = (double)bf16_round((float)gd);
-          }
-        }
+        gradient(i, j, ix, key[i], gext, &g, &gd);
         X[ix] = std::fmaf(-r, g, X[ix]);     // y = x - eta G / sqrt(.)
         B2[ix] = std::fmaf(g, g, B2[ix]);    // A^2 = B^2 + G o G
         Xd[ix] = Xd[ix] - etd * gd / std::sqrt(dd);
@@ -261,9 +279,75 @@ struct Oracle {
     }
   }
 
+  // One iteration of Algorithm 2 (Local SGD) without its averaging branch:
+  // y_{i,t} = x_{i,t-1} - eta G_{i,t}.  No accumulator is kept.
+  void local_sgd_step(const float* gext) {
+    t += 1;
+    tp += 1;
+    const float et = eta_t();
+    const double etd = eta_t_d();
+    const std::vector<uint64_t> key = step_keys();
+    for (uint64_t j = 0; j < n; ++j)
+      for (uint32_t i = 0; i < W; ++i) {
+        size_t ix = (size_t)i * n + j;
+        float g;
+        double gd;
+        gradient(i, j, ix, key[i], gext, &g, &gd);
+        X[ix] = std::fmaf(-et, g, X[ix]);
+        Xd[ix] = Xd[ix] - etd * gd;
+      }
+  }
+
+  // One iteration of Algorithm 1 (Distributed AdaGrad): every worker evaluates its gradient at
+  // the common iterate x_{t-1}; G_t = (1/n) sum_i G_{i,t}; B^2_t = B^2_{t-1} + G_t o G_t;
+  // x_t = x_{t-1} - eta G_t / sqrt(B^2_t + eps^2)  (the UPDATED accumulator).  All replicas
+  // stay equal; one gradient exchange per iteration is counted in nsync.
+  void adagrad_step(const float* gext) {
+    t += 1;
+    const float eps2 = eps * eps;
+    const float et = eta_t();
+    const double etd = eta_t_d();
+    const double eps2d = (double)eps * (double)eps;
+    const std::vector<uint64_t> key = step_keys();
+    std::vector<float> vg(W);
+    for (uint64_t j = 0; j < n; ++j) {
+      double gsum = 0;
+      for (uint32_t i = 0; i < W; ++i) {
+        float g;
+        double gd;
+        gradient(i, j, j /* replica 0 holds the common iterate */, key[i], gext, &g, &gd);
+        vg[i] = g;
+        gsum += gd;
+      }
+      float gm = tree_sum(vg) / (float)W;
+      double gmd = gsum / (double)W;
+      float b = std::fmaf(gm, gm, B2[j]);
+      float d = b + eps2;
+      float r = et / std::sqrt(d);
+      float x = std::fmaf(-r, gm, X[j]);
+      double bd = B2d[j] + gmd * gmd;
+      double xd = Xd[j] - etd * gmd / std::sqrt(bd + eps2d);
+      for (uint32_t i = 0; i < W; ++i) {
+        size_t ix = (size_t)i * n + j;
+        X[ix] = x; B2[ix] = b; Xd[ix] = xd; B2d[ix] = bd;
+      }
+      Bs[j] = b;
+      Bsd[j] = bd;
+    }
+    nsync += 1;
+  }
+
+  void local_step(const float* gext) {
+    if (rule == kRuleLocalSGD) local_sgd_step(gext);
+    else if (rule == kRuleAdaGrad) adagrad_step(gext);
+    else adaalter_step(gext);
+  }
+
   // Synchronisation branch of Algorithm 3: means of y and A^2 over workers
   // replace every worker's x and B^2; the mean B^2 becomes the stale denominator.
+  // (Algorithm 2's averaging branch is the same with the accumulator left out.)
   void sync() {
+    if (rule == kRuleLocalSGD) { sync_x_only(); return; }
     std::vector<float> vx(W), vb(W);
     std::vector<double> vxd(W), vbd(W);
     for (uint64_t j = 0; j < n; ++j) {
@@ -292,10 +376,28 @@ struct Oracle {
     nsync += 1;
   }
 
+  // Algorithm 2, else-branch: x_{i,t} = (1/n) sum_k y_{k,t}.
+  void sync_x_only() {
+    std::vector<float> vx(W);
+    for (uint64_t j = 0; j < n; ++j) {
+      for (uint32_t i = 0; i < W; ++i) vx[i] = X[(size_t)i * n + j];
+      float xm = tree_sum(vx) / (float)W;
+      double xs = 0;
+      for (uint32_t i = 0; i < W; ++i) xs += Xd[(size_t)i * n + j];
+      double xmd = xs / (double)W;
+      for (uint32_t i = 0; i < W; ++i) {
+        X[(size_t)i * n + j] = xm;
+        Xd[(size_t)i * n + j] = xmd;
+      }
+    }
+    tp = 0;
+    nsync += 1;
+  }
+
   void run(uint64_t T) {
     for (uint64_t k = 0; k < T; ++k) {
       local_step(nullptr);
-      if (tp == H) sync();
+      if (rule != kRuleAdaGrad && tp == H) sync();
     }
   }
 };
@@ -344,6 +446,7 @@ void ora_set_grad_constant(void* h, const float* s /* n or NULL => 1 */) {
 void ora_set_grad_bf16(void* h, int on) { ((Oracle*)h)->bf16 = on != 0; }
 void ora_set_identical_workers(void* h, int on) { ((Oracle*)h)->identical_workers = on != 0; }
 void ora_set_warmup(void* h, uint32_t steps) { ((Oracle*)h)->warm_up_steps = steps; }
+void ora_set_rule(void* h, int rule) { ((Oracle*)h)->rule = rule; }
 
 void ora_local_step(void* h) { ((Oracle*)h)->local_step(nullptr); }
 void ora_local_step_grads(void* h, const float* g /* [W][n] */) { ((Oracle*)h)->local_step(g); }

@@ -61,6 +61,7 @@ def lib() -> C.CDLL:
             L.ora_set_grad_bf16.argtypes = [vp, C.c_int]
             L.ora_set_identical_workers.argtypes = [vp, C.c_int]
             L.ora_set_warmup.argtypes = [vp, u32]
+            L.ora_set_rule.argtypes = [vp, C.c_int]
             L.ora_local_step.argtypes = [vp]
             L.ora_local_step_grads.argtypes = [vp, vp]
             L.ora_sync.argtypes = [vp]
@@ -140,6 +141,10 @@ class Oracle:
 
     def set_warmup(self, steps):
         self.L.ora_set_warmup(self.h, int(steps))
+
+    def set_rule(self, rule):
+        """0 = Local AdaAlter (Algorithm 3), 1 = Local SGD (Algorithm 2), 2 = Distributed AdaGrad (Algorithm 1)."""
+        self.L.ora_set_rule(self.h, int(rule))
 
     # ---- schedule ----------------------------------------------------------
     def local_step(self, grads=None):
