@@ -49,6 +49,9 @@ enum {
 enum { LA_F32 = 0, LA_BF16 = 1 };               /* gradient dtype */
 enum { LA_FUSE_NONE = 0, LA_FUSE_STEP_SYNC = 1, /* la_run: step t'=H and its sync in one pass */
        LA_FUSE_SYNC_STEP = 2 };                 /* la_run: sync folded into the following step */
+enum { LA_RULE_ADAALTER = 0,  /* Algorithm 3, Local AdaAlter (default) */
+       LA_RULE_LOCAL_SGD = 1, /* Algorithm 2: y = x - eta G, x averaged every H steps, no accumulator */
+       LA_RULE_ADAGRAD = 2 }; /* Algorithm 1: gradients averaged every step, B^2 += G o G, updated B^2 divides */
 #define LA_H_NEVER 0xFFFFFFFFu                  /* H = +infinity: never synchronise */
 #define LA_MAX_WORKERS 64u
 
@@ -111,6 +114,12 @@ int la_set_grad_dtype(la_ctx* ctx, int dtype);
 int la_set_identical_workers(la_ctx* ctx, int on);
 /* Warm-up of Section 6.2: eta_t = eta * min(1, t / warm_up_steps); 0 switches it off. */
 int la_set_warmup(la_ctx* ctx, uint32_t warm_up_steps);
+/* Baseline update rules of the paper in the same sweep (LA_RULE_*): Local SGD (Algorithm 2) and
+ * Distributed AdaGrad (Algorithm 1), for fp32 generated gradients.  Only legal while t' == 0.
+ * AdaGrad keeps ONE shared iterate (all workers see x_{t-1}); W only sets how many gradients are
+ * averaged per step; la_read_state returns that iterate for any worker, la_sync is LA_ESTATE,
+ * and n_sync counts one gradient exchange per iteration. */
+int la_set_rule(la_ctx* ctx, int rule);
 /* How la_run realises the synchronisation (LA_FUSE_*); results are bitwise the same. */
 int la_set_fusion(la_ctx* ctx, int mode);
 /* Tuning knob: the sweep kernels run as a grid-stride loop over at most

@@ -16,21 +16,21 @@
 
 namespace la {
 
-SweepKernel lookup_sweep_w0(int, bool, bool, bool, bool);
-SweepKernel lookup_sweep_w1(int, bool, bool, bool, bool);
-SweepKernel lookup_sweep_w2(int, bool, bool, bool, bool);
-SweepKernel lookup_sweep_w4(int, bool, bool, bool, bool);
-SweepKernel lookup_sweep_w8(int, bool, bool, bool, bool);
-SweepKernel lookup_sweep_w16(int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w0(int, int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w1(int, int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w2(int, int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w4(int, int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w8(int, int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w16(int, int, bool, bool, bool, bool);
 
-SweepKernel lookup_sweep(int W, int gm, bool bf16, bool pre, bool step, bool post) {
+SweepKernel lookup_sweep(int W, int rule, int gm, bool bf16, bool pre, bool step, bool post) {
   switch (W) {
-    case 1: return lookup_sweep_w1(gm, bf16, pre, step, post);
-    case 2: return lookup_sweep_w2(gm, bf16, pre, step, post);
-    case 4: return lookup_sweep_w4(gm, bf16, pre, step, post);
-    case 8: return lookup_sweep_w8(gm, bf16, pre, step, post);
-    case 16: return lookup_sweep_w16(gm, bf16, pre, step, post);
-    default: return lookup_sweep_w0(gm, bf16, pre, step, post);
+    case 1: return lookup_sweep_w1(rule, gm, bf16, pre, step, post);
+    case 2: return lookup_sweep_w2(rule, gm, bf16, pre, step, post);
+    case 4: return lookup_sweep_w4(rule, gm, bf16, pre, step, post);
+    case 8: return lookup_sweep_w8(rule, gm, bf16, pre, step, post);
+    case 16: return lookup_sweep_w16(rule, gm, bf16, pre, step, post);
+    default: return lookup_sweep_w0(rule, gm, bf16, pre, step, post);
   }
 }
 
@@ -73,6 +73,7 @@ struct la_ctx {
   bool bf16 = false, identical = false;
   uint64_t seed = 0;
   int fusion = LA_FUSE_NONE;
+  int rule = LA_RULE_ADAALTER;
   bool profiling = false;
   int device = 0;
   cudaStream_t stream = nullptr;
@@ -193,6 +194,20 @@ int begin_timed(la_ctx* c, int cls, EventPair* ep) {
 // every replica's x and B^2 read and written once, worker-independent arrays once.
 double pass_bytes(const la_ctx* c, bool pre, bool step, bool post, int gm) {
   const double n = (double)c->N, W = (double)c->W;
+  if (c->rule == LA_RULE_ADAGRAD) {                 // one shared x, B2: read + write, Bs written
+    double b = 20.0 * n;
+    if (gm == la::kGradQuadratic) b += 8.0 * n;
+    if (gm == la::kGradNoiseScaled || (gm == la::kGradConstant && c->has_s)) b += 4.0 * n;
+    return b;
+  }
+  if (c->rule == LA_RULE_LOCAL_SGD) {               // X only: read + write
+    double b = 8.0 * W * n;
+    if (step) {
+      if (gm == la::kGradQuadratic) b += 8.0 * n;
+      if (gm == la::kGradNoiseScaled || (gm == la::kGradConstant && c->has_s)) b += 4.0 * n;
+    }
+    return b;
+  }
   double b = 16.0 * W * n;                          // X, B2: read + write
   if (pre || post) b += 4.0 * n;                    // stale accumulator written
   if (step && !pre) b += 4.0 * n;                   // stale accumulator read
@@ -206,9 +221,12 @@ double pass_bytes(const la_ctx* c, bool pre, bool step, bool post, int gm) {
 }
 
 int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t tp, int gm, const void* gext) {
-  const la::SweepKernel k = la::lookup_sweep((int)c->W, gm, c->bf16 && gm <= la::kGradQuadratic, pre, step, post);
+  const la::SweepKernel k =
+      la::lookup_sweep((int)c->W, c->rule, gm, c->bf16 && gm <= la::kGradQuadratic, pre, step, post);
   la::SweepFn fn = k.fn;
-  if (!fn) return fail(c, LA_ESTATE, "no kernel for this combination (W=%u grad=%d)", c->W, gm);
+  if (!fn)
+    return fail(c, LA_ESTATE, "no kernel for this combination (W=%u rule=%d grad=%d bf16=%d)", c->W, c->rule, gm,
+                (int)c->bf16);
   la::SweepParams p{};
   p.X = c->X; p.B2 = c->B2; p.Bs = c->Bs;
   p.a = c->pa; p.c = c->pc; p.s = c->has_s ? c->ps : nullptr;
@@ -439,6 +457,15 @@ int la_set_fusion(la_ctx* c, int mode) {
   return LA_OK;
 }
 
+int la_set_rule(la_ctx* c, int rule) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (rule != LA_RULE_ADAALTER && rule != LA_RULE_LOCAL_SGD && rule != LA_RULE_ADAGRAD)
+    return fail(c, LA_EINVAL, "unknown update rule %d", rule);
+  if (c->tp != 0) return fail(c, LA_ESTATE, "the update rule can only change right after a synchronisation (t' = 0)");
+  c->rule = rule;
+  return LA_OK;
+}
+
 int la_set_profiling(la_ctx* c, int on) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   DeviceGuard guard(c->device);
@@ -460,7 +487,9 @@ int la_local_step(la_ctx* c) {
   DeviceGuard guard(c->device);
   int rc = launch_sweep(c, false, true, false, c->t + 1, c->tp + 1, c->grad_kind, nullptr);
   if (rc) return rc;
-  c->t += 1; c->tp += 1;
+  c->t += 1;
+  if (c->rule == LA_RULE_ADAGRAD) c->nsync += 1;  // Algorithm 1 exchanges gradients every iteration
+  else c->tp += 1;
   return LA_OK;
 }
 
@@ -468,6 +497,7 @@ int la_local_step_grads(la_ctx* c, const void* g_dev, int dtype) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   if (!g_dev) return fail(c, LA_EINVAL, "g_dev is NULL");
   if (dtype != LA_F32 && dtype != LA_BF16) return fail(c, LA_EINVAL, "dtype must be LA_F32 or LA_BF16");
+  if (c->rule != LA_RULE_ADAALTER) return fail(c, LA_ESTATE, "supplied gradients are implemented for Local AdaAlter only");
   DeviceGuard guard(c->device);
   int rc = launch_sweep(c, false, true, false, c->t + 1, c->tp + 1,
                         dtype == LA_F32 ? la::kGradExternalF32 : la::kGradExternalBF16, g_dev);
@@ -478,6 +508,7 @@ int la_local_step_grads(la_ctx* c, const void* g_dev, int dtype) {
 
 int la_sync(la_ctx* c) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (c->rule == LA_RULE_ADAGRAD) return fail(c, LA_ESTATE, "Distributed AdaGrad keeps one shared iterate: nothing to synchronise");
   DeviceGuard guard(c->device);
   int rc = launch_sweep(c, true, false, false, c->t, 0, la::kGradNoise, nullptr);
   if (rc) return rc;
@@ -490,6 +521,13 @@ int la_run(la_ctx* c, uint64_t T) {
   DeviceGuard guard(c->device);
   // Algorithm 3: for t in [T]: local step; if mod(t, H) == 0 (tracked as t' == H): synchronise.
   // `deferred` marks a synchronisation that is due but has been folded into the next step.
+  if (c->rule == LA_RULE_ADAGRAD) {  // Algorithm 1: every iteration is one fully synchronous pass
+    for (uint64_t k = 0; k < T; ++k) {
+      int rc = la_local_step(c);
+      if (rc) return rc;
+    }
+    return LA_OK;
+  }
   bool deferred = false;
   for (uint64_t k = 0; k < T; ++k) {
     int rc;
@@ -525,6 +563,7 @@ int la_read_range(la_ctx* c, uint32_t worker, uint64_t j0, uint64_t n, float* x_
   if (worker >= c->W) return fail(c, LA_EINVAL, "worker %u out of range (W=%u)", worker, c->W);
   if (j0 > c->N || n > c->N - j0) return fail(c, LA_EINVAL, "coordinate range out of bounds");
   DeviceGuard guard(c->device);
+  if (c->rule == LA_RULE_ADAGRAD) worker = 0;  // one shared iterate (Algorithm 1)
   const size_t bytes = n * sizeof(float);
   if (n) {
     if (x_host) LA_CUDA(c, cudaMemcpyAsync(x_host, c->X + (uint64_t)worker * c->stride + j0, bytes, cudaMemcpyDeviceToHost, c->stream));

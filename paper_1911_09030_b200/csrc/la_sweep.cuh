@@ -140,25 +140,27 @@ __device__ __forceinline__ Vec<V> div_by_workers(const Vec<V>& a, uint32_t W) {
 // like the carries of a binary counter.  After pushing worker i the two top entries are
 // merged once for every trailing zero bit of (i+1); left operand = older entry.  With W known
 // at compile time the loop unrolls and every stack index is a constant (registers only).
-template <int V>
+// ACC = false drops the accumulator component (Local SGD averages x only; AdaGrad averages
+// gradients).
+template <int V, bool ACC = true>
 struct PairTree {
-  Vec<V> x[kTreeDepth], b[kTreeDepth];
+  Vec<V> x[kTreeDepth], b[ACC ? kTreeDepth : 1];
   int sp = 0;
   __device__ __forceinline__ void push(uint32_t i, const Vec<V>& vx, const Vec<V>& vb) {
     x[sp] = vx;
-    b[sp] = vb;
+    if (ACC) b[ACC ? sp : 0] = vb;
     ++sp;
     for (uint32_t cnt = i + 1u; (cnt & 1u) == 0u; cnt >>= 1) {
       --sp;
       x[sp - 1] = add(x[sp - 1], x[sp]);
-      b[sp - 1] = add(b[sp - 1], b[sp]);
+      if (ACC) b[ACC ? sp - 1 : 0] = add(b[ACC ? sp - 1 : 0], b[ACC ? sp : 0]);
     }
   }
   __device__ __forceinline__ void finish() {
     while (sp > 1) {
       --sp;
       x[sp - 1] = add(x[sp - 1], x[sp]);
-      b[sp - 1] = add(b[sp - 1], b[sp]);
+      if (ACC) b[ACC ? sp - 1 : 0] = add(b[ACC ? sp - 1 : 0], b[ACC ? sp : 0]);
     }
   }
 };
@@ -190,24 +192,24 @@ struct ReplicaChunk {
 
 // Loads replicas i0 .. i0+CH-1; `addr` is the address of x of replica i0 for this coordinate
 // group and is left pointing at replica i0+CH.  B^2 of a replica sits `b_delta` bytes after x.
-template <int V, int CH>
+template <int V, int CH, bool ACC = true>
 __device__ __forceinline__ void load_chunk(ReplicaChunk<V, CH>& ch, uint64_t& addr, uint64_t b_delta,
                                            uint64_t stride_bytes, uint32_t W, uint32_t i0) {
 #pragma unroll
   for (int k = 0; k < CH; ++k)
     if (i0 + k < W) {
       ch.x[k] = ld_stream<V>(as_ptr(addr));
-      ch.b[k] = ld_stream<V>(as_ptr(addr + b_delta));
+      if (ACC) ch.b[k] = ld_stream<V>(as_ptr(addr + b_delta));
       advance(addr, stride_bytes);
     }
 }
 
 // Stores x and B^2 of one replica at `addr` and advances to the next replica.
-template <int V>
+template <int V, bool ACC = true>
 __device__ __forceinline__ void store_replica(uint64_t& addr, uint64_t b_delta, uint64_t stride_bytes,
                                               const Vec<V>& x, const Vec<V>& b) {
   st_stream<V>(as_mut(addr), x);
-  st_stream<V>(as_mut(addr + b_delta), b);
+  if (ACC) st_stream<V>(as_mut(addr + b_delta), b);
   advance(addr, stride_bytes);
 }
 
@@ -264,16 +266,18 @@ __device__ __forceinline__ Vec<V> gradient(const SweepParams& p, const CoordInpu
 }
 
 // y = x - r g ; A^2 = B^2 + g g   (Algorithm 3), one fused multiply-add each.
-template <int V>
+template <int V, bool ACC = true>
 __device__ __forceinline__ void apply(const Vec<V>& r, const Vec<V>& g, Vec<V>& x, Vec<V>& b) {
 #pragma unroll
   for (int k = 0; k < V; ++k) {
     x.v[k] = __fmaf_rn(-r.v[k], g.v[k], x.v[k]);
-    b.v[k] = __fmaf_rn(g.v[k], g.v[k], b.v[k]);
+    if (ACC) b.v[k] = __fmaf_rn(g.v[k], g.v[k], b.v[k]);
   }
 }
 
-template <int W_, int V, int GM, bool BF16, bool PRE, bool STEP, bool POST, int MINB>
+// ACC = true: Algorithm 3 (Local AdaAlter).  ACC = false: Algorithm 2 (Local SGD) — the same sweep
+// without accumulators: y = x - eta_t G, and the synchronisation averages x only.
+template <int W_, int V, int GM, bool BF16, bool PRE, bool STEP, bool POST, int MINB, bool ACC = true>
 __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) {
   static_assert(!(PRE && POST), "one synchronisation per pass");
   static_assert(V == 2 || V == 4, "a thread owns 2 or 4 coordinates");
@@ -309,7 +313,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
   const uint64_t nthreads = (uint64_t)gridDim.x * blockDim.x;
   uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (grp >= ngroups) return;
-  constexpr bool kLoadsBs = STEP && !PRE;
+  constexpr bool kLoadsBs = STEP && !PRE && ACC;
 
   const uint64_t x_base = reinterpret_cast<uint64_t>(p.X);
   const uint64_t b_delta = reinterpret_cast<uint64_t>(p.B2) - x_base;
@@ -319,7 +323,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
   CoordInputs<V> in_next;
   load_coord<GM, STEP, kLoadsBs, V>(in_next, p, grp * V);
   uint64_t ld_addr = x_base + grp * (V * sizeof(float));
-  load_chunk<V, CH>(nxt, ld_addr, b_delta, stride_bytes, W, 0u);
+  load_chunk<V, CH, ACC>(nxt, ld_addr, b_delta, stride_bytes, W, 0u);
 
   for (;;) {
     const uint64_t off = grp * V;
@@ -331,17 +335,18 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
 
     Vec<V> r;
     if (kLoadsBs) r = step_size<V>(in.bs, q, eta_t);
-    PairTree<V> tree;
+    if (!ACC) r = splat<V>(eta_t);
+    PairTree<V, ACC> tree;
 
 #pragma unroll kOuterUnroll
     for (uint32_t i0 = 0; i0 < W; i0 += CH) {
       ReplicaChunk<V, CH> cur = nxt;
       if (i0 + CH < W) {
-        load_chunk<V, CH>(nxt, ld_addr, b_delta, stride_bytes, W, i0 + CH);
+        load_chunk<V, CH, ACC>(nxt, ld_addr, b_delta, stride_bytes, W, i0 + CH);
       } else if (has_next) {
         load_coord<GM, STEP, kLoadsBs, V>(in_next, p, next_grp * V);
         ld_addr = x_base + next_grp * (V * sizeof(float));
-        load_chunk<V, CH>(nxt, ld_addr, b_delta, stride_bytes, W, 0u);
+        load_chunk<V, CH, ACC>(nxt, ld_addr, b_delta, stride_bytes, W, 0u);
       }
       asm volatile("" ::: "memory");
 #pragma unroll
@@ -352,11 +357,11 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
             tree.push(i, cur.x[k], cur.b[k]);
           } else {
             const Vec<V> g = gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
-            apply<V>(r, g, cur.x[k], cur.b[k]);
+            apply<V, ACC>(r, g, cur.x[k], cur.b[k]);
             if (POST) {
               tree.push(i, cur.x[k], cur.b[k]);
             } else {
-              store_replica<V>(st_addr, b_delta, stride_bytes, cur.x[k], cur.b[k]);
+              store_replica<V, ACC>(st_addr, b_delta, stride_bytes, cur.x[k], cur.b[k]);
             }
           }
         }
@@ -367,25 +372,77 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
       // also the new stale denominator
       tree.finish();
       const Vec<V> xm = div_by_workers<W_, V>(tree.x[0], W);
-      const Vec<V> bm = div_by_workers<W_, V>(tree.b[0], W);
-      st_stream<V>(p.Bs + off, bm);
+      Vec<V> bm = xm;
+      if (ACC) {
+        bm = div_by_workers<W_, V>(tree.b[0], W);
+        st_stream<V>(p.Bs + off, bm);
+      }
       if (PRE && STEP) {
         // first step of the next period: every replica starts from the mean, t' = 1
-        r = step_size<V>(bm, q, eta_t);
+        if (ACC) r = step_size<V>(bm, q, eta_t);
 #pragma unroll kOuterUnroll
         for (uint32_t i = 0; i < W; ++i) {
           Vec<V> xv = xm, bv = bm;
           const Vec<V> g = gradient<GM, BF16, V>(p, in, xv, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
-          apply<V>(r, g, xv, bv);
-          store_replica<V>(st_addr, b_delta, stride_bytes, xv, bv);
+          apply<V, ACC>(r, g, xv, bv);
+          store_replica<V, ACC>(st_addr, b_delta, stride_bytes, xv, bv);
         }
       } else {
 #pragma unroll kOuterUnroll
-        for (uint32_t i = 0; i < W; ++i) store_replica<V>(st_addr, b_delta, stride_bytes, xm, bm);
+        for (uint32_t i = 0; i < W; ++i) store_replica<V, ACC>(st_addr, b_delta, stride_bytes, xm, bm);
       }
     }
     if (!has_next) break;
     grp = next_grp;
+  }
+}
+
+// Algorithm 1 (Distributed AdaGrad), one iteration: every worker's gradient at the COMMON iterate,
+// G_t = mean over workers (same adjacent-pair tree), B^2_t = B^2_{t-1} + G_t o G_t,
+// x_t = x_{t-1} - eta_t G_t / sqrt(B^2_t + eps^2) with the UPDATED accumulator.  The iterate is
+// shared by construction, so only replica 0 is kept; the accumulator is mirrored into Bs.
+template <int W_, int V, int GM, int MINB>
+__global__ void __launch_bounds__(LA_BLOCK, MINB) la_adagrad(const SweepParams p) {
+  constexpr bool kNeedsNoise = (GM == kGradNoise || GM == kGradNoiseScaled || GM == kGradQuadratic);
+  constexpr int kOuterUnroll = (W_ > 0) ? kMaxWorkers : 1;
+  const uint32_t W = (W_ > 0) ? (uint32_t)W_ : p.W;
+  __shared__ uint64_t keys[kMaxWorkers];
+  if (kNeedsNoise) {
+    if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, p.t, p.identical_workers ? 0u : threadIdx.x);
+    __syncthreads();
+  }
+  const float eps2 = __fmul_rn(p.eps, p.eps);
+  float eta_t = p.eta;
+  if (p.warm_up_steps != 0u) {
+    const float ratio = __fdiv_rn(__ull2float_rn(p.t), __uint2float_rn(p.warm_up_steps));
+    eta_t = __fmul_rn(p.eta, fminf(1.0f, ratio));
+  }
+  const uint64_t ngroups = (p.n + (uint64_t)(V - 1)) / (uint64_t)V;
+  const uint64_t nthreads = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < ngroups; grp += nthreads) {
+    const uint64_t off = grp * V;
+    CoordInputs<V> in;
+    load_coord<GM, true, false, V>(in, p, off);
+    Vec<V> x = ld_stream<V>(p.X + off);
+    Vec<V> b = ld_stream<V>(p.B2 + off);
+    const uint64_t ctr0 = kGoldenGamma * (((p.j_base + off) >> 1) + 1u);
+    PairTree<V, false> tree;
+#pragma unroll kOuterUnroll
+    for (uint32_t i = 0; i < W; ++i) {
+      const Vec<V> g = gradient<GM, false, V>(p, in, x, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
+      tree.push(i, g, g);
+    }
+    tree.finish();
+    const Vec<V> gm = div_by_workers<W_, V>(tree.x[0], W);
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+      b.v[k] = __fmaf_rn(gm.v[k], gm.v[k], b.v[k]);
+      const float r = __fdiv_rn(eta_t, __fsqrt_rn(__fadd_rn(b.v[k], eps2)));
+      x.v[k] = __fmaf_rn(-r, gm.v[k], x.v[k]);
+    }
+    st_stream<V>(p.X + off, x);
+    st_stream<V>(p.B2 + off, b);
+    st_stream<V>(p.Bs + off, b);
   }
 }
 
@@ -395,6 +452,7 @@ struct SweepKernel {
   SweepFn fn;
   int vec;
 };
-SweepKernel lookup_sweep(int W, int gm, bool bf16, bool pre, bool step, bool post);
+// rule: 0 = Local AdaAlter, 1 = Local SGD, 2 = Distributed AdaGrad (one kernel per step)
+SweepKernel lookup_sweep(int W, int rule, int gm, bool bf16, bool pre, bool step, bool post);
 
 }  // namespace la

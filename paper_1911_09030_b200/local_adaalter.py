@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_HERE, "liblocal_adaalter.so")
 LA_OK, LA_EINVAL, LA_ENOMEM, LA_ECUDA, LA_ESTATE = 0, -1, -2, -3, -4
 LA_F32, LA_BF16 = 0, 1
 LA_FUSE_NONE, LA_FUSE_STEP_SYNC, LA_FUSE_SYNC_STEP = 0, 1, 2
+LA_RULE_ADAALTER, LA_RULE_LOCAL_SGD, LA_RULE_ADAGRAD = 0, 1, 2
 LA_H_NEVER = 0xFFFFFFFF
 LA_MAX_WORKERS = 64
 
@@ -62,6 +63,7 @@ def lib() -> C.CDLL:
             "la_set_identical_workers": [vp, i32],
             "la_set_warmup": [vp, u32],
             "la_set_fusion": [vp, i32],
+            "la_set_rule": [vp, i32],
             "la_set_launch_shape": [vp, i32],
             "la_set_profiling": [vp, i32],
             "la_local_step": [vp],
@@ -214,6 +216,9 @@ class LocalAdaAlter:
 
     def set_warmup(self, steps):
         self._ck(self.L.la_set_warmup(self.h, int(steps)))
+
+    def set_rule(self, rule):
+        self._ck(self.L.la_set_rule(self.h, int(rule)))
 
     def set_fusion(self, mode):
         self._ck(self.L.la_set_fusion(self.h, int(mode)))
