@@ -166,6 +166,41 @@ int la_set_counters(la_ctx* ctx, uint64_t t, uint32_t t_prime, uint64_t n_sync);
  * reset != 0 clears the counters after reading. */
 int la_get_stats(la_ctx* ctx, la_stats* out, int reset);
 
+/* ---- sharding BY WORKER across GPUs (one process per GPU) -----------------------------------
+ * The layout of the paper: the workers of Algorithm 3 sit on different devices and exchange x
+ * and B^2 every H steps (Section 4.2).  A rank holds W (local) replicas out of W_total.
+ * The synchronisation is three enqueued phases around a library-owned exchange buffer
+ * [2][stride] (sums of x, sums of B^2); the HOST orders them (la_stream_sync + a barrier across
+ * ranks between phases); no kernel ever waits for another rank:
+ *   la_comm_export   buffer <- adjacent-pair tree sum over the local replicas
+ *   la_comm_combine  this rank's coordinate slice: adjacent-pair tree over all ranks' buffers in
+ *                    rank order (plain peer loads), total stored into EVERY rank's buffer
+ *                    (alternatively the caller all-reduces the buffer itself, e.g. with NCCL)
+ *   la_comm_import   x, B^2 of every local replica <- total / W_total; stale <- mean B^2;
+ *                    t' = 0; n_sync += 1
+ * With W a power of two the result equals the single-GPU la_sync over W_total replicas bit for
+ * bit (a caller-side all-reduce gives the same means up to its summation order).  Local
+ * AdaAlter rule only. */
+/* Global index of local replica 0 and the total worker count: the noise of local replica i is
+ * that of worker worker_base + i.  W_total = 0 returns to the unsharded numbering. */
+int la_set_worker_range(la_ctx* ctx, uint32_t worker_base, uint32_t W_total);
+/* Allocate the exchange buffer (freed by la_destroy) and fix this context's rank.  If no worker
+ * range was set: worker_base = rank * W, W_total = world * W. */
+int la_comm_create(la_ctx* ctx, uint32_t rank, uint32_t world);
+/* Device pointer and size of the exchange buffer (2 * stride floats). */
+int la_comm_buffer(la_ctx* ctx, void** dev_ptr, uint64_t* bytes);
+/* 64-byte CUDA IPC handle of the exchange buffer, to be sent to the other ranks (host buffer). */
+int la_comm_ipc_handle(la_ctx* ctx, void* handle64_host);
+/* Attach rank peer_rank's exchange buffer: from its IPC handle (another process), or as a raw
+ * device pointer that is already valid here (same process).  Mappings are closed by la_destroy. */
+int la_comm_open_peer(la_ctx* ctx, uint32_t peer_rank, const void* handle64_host);
+int la_comm_set_peer(la_ctx* ctx, uint32_t peer_rank, void* dev_ptr);
+int la_comm_export(la_ctx* ctx);
+int la_comm_combine(la_ctx* ctx);
+int la_comm_import(la_ctx* ctx);
+/* Block until the context's stream is idle. */
+int la_stream_sync(la_ctx* ctx);
+
 #ifdef __cplusplus
 }
 #endif

@@ -192,6 +192,7 @@ struct Oracle {
   float sigma = 0;
   bool bf16 = false;
   bool identical_workers = false;
+  uint32_t worker_base = 0;    // global index of local worker 0 (workers sharded over ranks)
   std::vector<float> a, c, s;  // s empty => s == 1
   // state, fp32
   std::vector<float> X, B2, Bs;  // X,B2: [W][n]; Bs: [n]
@@ -246,7 +247,7 @@ struct Oracle {
 
   std::vector<uint64_t> step_keys() const {
     std::vector<uint64_t> key(W);
-    for (uint32_t i = 0; i < W; ++i) key[i] = stream_key(seed, t, identical_workers ? 0u : i);
+    for (uint32_t i = 0; i < W; ++i) key[i] = stream_key(seed, t, identical_workers ? 0u : worker_base + i);
     return key;
   }
 
@@ -447,6 +448,7 @@ void ora_set_grad_bf16(void* h, int on) { ((Oracle*)h)->bf16 = on != 0; }
 void ora_set_identical_workers(void* h, int on) { ((Oracle*)h)->identical_workers = on != 0; }
 void ora_set_warmup(void* h, uint32_t steps) { ((Oracle*)h)->warm_up_steps = steps; }
 void ora_set_rule(void* h, int rule) { ((Oracle*)h)->rule = rule; }
+void ora_set_worker_base(void* h, uint32_t base) { ((Oracle*)h)->worker_base = base; }
 
 void ora_local_step(void* h) { ((Oracle*)h)->local_step(nullptr); }
 void ora_local_step_grads(void* h, const float* g /* [W][n] */) { ((Oracle*)h)->local_step(g); }

@@ -62,6 +62,7 @@ def lib() -> C.CDLL:
             L.ora_set_identical_workers.argtypes = [vp, C.c_int]
             L.ora_set_warmup.argtypes = [vp, u32]
             L.ora_set_rule.argtypes = [vp, C.c_int]
+            L.ora_set_worker_base.argtypes = [vp, u32]
             L.ora_local_step.argtypes = [vp]
             L.ora_local_step_grads.argtypes = [vp, vp]
             L.ora_sync.argtypes = [vp]
@@ -141,6 +142,10 @@ class Oracle:
 
     def set_warmup(self, steps):
         self.L.ora_set_warmup(self.h, int(steps))
+
+    def set_worker_base(self, base):
+        """Noise of local worker i is that of global worker base + i."""
+        self.L.ora_set_worker_base(self.h, int(base))
 
     def set_rule(self, rule):
         """0 = Local AdaAlter (Algorithm 3), 1 = Local SGD (Algorithm 2), 2 = Distributed AdaGrad (Algorithm 1)."""

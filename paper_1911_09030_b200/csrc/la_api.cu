@@ -12,6 +12,7 @@
 #include <vector>
 
 #include "../../include/local_adaalter.h"
+#include "la_exchange.cuh"
 #include "la_sweep.cuh"
 
 namespace la {
@@ -34,6 +35,25 @@ SweepKernel lookup_sweep(int W, int rule, int gm, bool bf16, bool pre, bool step
   }
 }
 
+ExchangeFn lookup_export_w0();
+ExchangeFn lookup_export_w1();
+ExchangeFn lookup_export_w2();
+ExchangeFn lookup_export_w4();
+ExchangeFn lookup_export_w8();
+ExchangeFn lookup_export_w16();
+
+ExchangeFn lookup_export(int W) {
+  switch (W) {
+    case 1: return lookup_export_w1();
+    case 2: return lookup_export_w2();
+    case 4: return lookup_export_w4();
+    case 8: return lookup_export_w8();
+    case 16: return lookup_export_w16();
+    default: return lookup_export_w0();
+  }
+}
+constexpr int kExchangeVec = 2;  // coordinates per thread in the exchange kernels
+
 __global__ void la_fill(float* X, float* B2, float* Bs, const float* x0, float b0sq, uint64_t stride,
                         uint64_t n, uint32_t W) {
   const uint64_t nthreads = (uint64_t)gridDim.x * blockDim.x;
@@ -52,6 +72,7 @@ __global__ void la_fill(float* X, float* B2, float* Bs, const float* x0, float b
 namespace {
 
 thread_local std::string g_create_error;
+constexpr uint64_t kExchangeVecHost = la::kExchangeVec;
 
 enum KernelClass { kClassLocal = 0, kClassSync = 1, kClassFused = 2, kClassOther = 3 };
 
@@ -84,6 +105,11 @@ struct la_ctx {
   bool owns_arena = false;
   float *X = nullptr, *B2 = nullptr, *Bs = nullptr, *pa = nullptr, *pc = nullptr, *ps = nullptr;
   bool has_s = false;
+  // sharding by worker: exchange buffer [2][stride], peers' buffers, global worker numbering
+  uint32_t worker_base = 0, W_total = 0, rank = 0, world = 1;
+  float* S = nullptr;
+  float* peerS[la::kMaxRanks] = {};
+  void* ipc_opened[la::kMaxRanks] = {};
   // schedule (Algorithm 3): t = local steps so far, tp = local steps since the last sync
   uint64_t t = 0, nsync = 0;
   uint32_t tp = 0;
@@ -234,6 +260,7 @@ int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t
   p.n = c->N; p.stride = c->stride; p.j_base = c->j_base;
   p.seed = c->seed; p.t = t; p.W = c->W; p.tp = tp;
   p.warm_up_steps = c->warm_up_steps; p.identical_workers = c->identical ? 1u : 0u;
+  p.worker_base = c->worker_base;
   p.eta = c->eta; p.eps = c->eps; p.sigma = c->sigma;
   const unsigned block = la::kBlockThreads;
   const uint64_t ngroups = (c->N + (uint64_t)k.vec - 1) / (uint64_t)k.vec;
@@ -379,6 +406,8 @@ void la_destroy(la_ctx* c) {
   cudaStreamSynchronize(c->stream);
   for (auto& p : c->pending) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
   for (auto& p : c->pool) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
+  for (auto*& m : c->ipc_opened) if (m) { cudaIpcCloseMemHandle(m); m = nullptr; }
+  if (c->S) cudaFree(c->S);
   if (c->owns_arena && c->arena) cudaFree(c->arena);
   delete c;
 }
@@ -621,6 +650,145 @@ int la_get_stats(la_ctx* c, la_stats* out, int reset) {
   if (rc) return rc;
   *out = c->stats;
   if (reset) c->stats = la_stats{};
+  return LA_OK;
+}
+
+// ---- sharding by worker -------------------------------------------------------------------
+int la_set_worker_range(la_ctx* c, uint32_t worker_base, uint32_t W_total) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (W_total == 0) { c->worker_base = 0; c->W_total = 0; return LA_OK; }
+  if ((uint64_t)worker_base + c->W > W_total) return fail(c, LA_EINVAL, "worker range exceeds W_total");
+  c->worker_base = worker_base; c->W_total = W_total;
+  return LA_OK;
+}
+
+int la_comm_create(la_ctx* c, uint32_t rank, uint32_t world) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (world == 0 || world > la::kMaxRanks || rank >= world) return fail(c, LA_EINVAL, "need rank < world <= %d", la::kMaxRanks);
+  if (c->rule != LA_RULE_ADAALTER) return fail(c, LA_ESTATE, "sharding by worker is implemented for Local AdaAlter only");
+  DeviceGuard guard(c->device);
+  if (!c->S) {
+    cudaError_t e = cudaMalloc((void**)&c->S, 2 * c->stride * sizeof(float));
+    if (e != cudaSuccess) { c->S = nullptr; cudaGetLastError(); return fail(c, LA_ENOMEM, "cudaMalloc of the exchange buffer failed: %s", cudaGetErrorString(e)); }
+    LA_CUDA(c, cudaMemsetAsync(c->S, 0, 2 * c->stride * sizeof(float), c->stream));
+  }
+  c->rank = rank; c->world = world;
+  for (auto& q : c->peerS) q = nullptr;
+  c->peerS[rank] = c->S;
+  if (c->W_total == 0) { c->W_total = c->W * world; c->worker_base = c->W * rank; }
+  return LA_OK;
+}
+
+int la_comm_buffer(la_ctx* c, void** dev_ptr, uint64_t* bytes) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
+  if (dev_ptr) *dev_ptr = c->S;
+  if (bytes) *bytes = 2 * c->stride * sizeof(float);
+  return LA_OK;
+}
+
+int la_comm_ipc_handle(la_ctx* c, void* handle64) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
+  if (!handle64) return fail(c, LA_EINVAL, "handle buffer is NULL");
+  static_assert(sizeof(cudaIpcMemHandle_t) == 64, "IPC handle size");
+  DeviceGuard guard(c->device);
+  cudaIpcMemHandle_t h;
+  LA_CUDA(c, cudaIpcGetMemHandle(&h, c->S));
+  std::memcpy(handle64, &h, sizeof h);
+  return LA_OK;
+}
+
+int la_comm_set_peer(la_ctx* c, uint32_t peer_rank, void* dev_ptr) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
+  if (peer_rank >= c->world || peer_rank == c->rank || !dev_ptr) return fail(c, LA_EINVAL, "bad peer rank or pointer");
+  c->peerS[peer_rank] = (float*)dev_ptr;
+  return LA_OK;
+}
+
+int la_comm_open_peer(la_ctx* c, uint32_t peer_rank, const void* handle64) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
+  if (peer_rank >= c->world || peer_rank == c->rank || !handle64) return fail(c, LA_EINVAL, "bad peer rank or handle");
+  DeviceGuard guard(c->device);
+  cudaIpcMemHandle_t h;
+  std::memcpy(&h, handle64, sizeof h);
+  void* mapped = nullptr;
+  LA_CUDA(c, cudaIpcOpenMemHandle(&mapped, h, cudaIpcMemLazyEnablePeerAccess));
+  if (c->ipc_opened[peer_rank]) cudaIpcCloseMemHandle(c->ipc_opened[peer_rank]);
+  c->ipc_opened[peer_rank] = mapped;
+  c->peerS[peer_rank] = (float*)mapped;
+  return LA_OK;
+}
+
+static int exchange_params(la_ctx* c, la::ExchangeParams* p, bool need_peers) {
+  if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
+  std::memset(p, 0, sizeof *p);
+  for (uint32_t r = 0; r < c->world; ++r) {
+    if (need_peers && !c->peerS[r]) return fail(c, LA_ESTATE, "exchange buffer of rank %u not attached", r);
+    p->S[r] = c->peerS[r];
+  }
+  p->X = c->X; p->B2 = c->B2; p->Bs = c->Bs;
+  p->n = c->N; p->stride = c->stride;
+  const uint64_t units = c->stride / 64;
+  p->slice_lo = units * c->rank / c->world * 64;
+  p->slice_hi = units * (c->rank + 1) / c->world * 64;
+  p->W = c->W; p->W_total = c->W_total; p->rank = c->rank; p->world = c->world;
+  return LA_OK;
+}
+
+static unsigned exchange_grid(const la_ctx* c, uint64_t coords) {
+  const uint64_t groups = (coords + kExchangeVecHost - 1) / kExchangeVecHost;
+  uint64_t blocks = (groups + la::kBlockThreads - 1) / la::kBlockThreads;
+  const uint64_t cap = (uint64_t)c->num_sms * 4096;
+  if (blocks > cap) blocks = cap;
+  return blocks ? (unsigned)blocks : 1u;
+}
+
+int la_comm_export(la_ctx* c) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  DeviceGuard guard(c->device);
+  la::ExchangeParams p;
+  int rc = exchange_params(c, &p, false);
+  if (rc) return rc;
+  la::lookup_export((int)c->W)<<<exchange_grid(c, c->N), la::kBlockThreads, 0, c->stream>>>(p);
+  LA_CUDA(c, cudaGetLastError());
+  c->stats.launches_other++;
+  return LA_OK;
+}
+
+int la_comm_combine(la_ctx* c) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  DeviceGuard guard(c->device);
+  la::ExchangeParams p;
+  int rc = exchange_params(c, &p, true);
+  if (rc) return rc;
+  if (p.slice_hi > p.slice_lo) {
+    la::la_combine_sums<la::kExchangeVec><<<exchange_grid(c, p.slice_hi - p.slice_lo), la::kBlockThreads, 0, c->stream>>>(p);
+    LA_CUDA(c, cudaGetLastError());
+    c->stats.launches_other++;
+  }
+  return LA_OK;
+}
+
+int la_comm_import(la_ctx* c) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  DeviceGuard guard(c->device);
+  la::ExchangeParams p;
+  int rc = exchange_params(c, &p, false);
+  if (rc) return rc;
+  la::la_import_means<la::kExchangeVec><<<exchange_grid(c, c->N), la::kBlockThreads, 0, c->stream>>>(p);
+  LA_CUDA(c, cudaGetLastError());
+  c->stats.launches_other++;
+  c->tp = 0; c->nsync += 1;
+  return LA_OK;
+}
+
+int la_stream_sync(la_ctx* c) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  DeviceGuard guard(c->device);
+  LA_CUDA(c, cudaStreamSynchronize(c->stream));
   return LA_OK;
 }
 

@@ -49,6 +49,7 @@ struct SweepParams {
   uint32_t tp;         // t' of the STEP part (local steps since the last sync, incl. this one)
   uint32_t warm_up_steps;
   uint32_t identical_workers;
+  uint32_t worker_base;  // global index of local replica 0 (sharding by worker); keys use worker_base + i
   float eta, eps, sigma;
 };
 
@@ -289,7 +290,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
 
   __shared__ uint64_t keys[kMaxWorkers];
   if (kNeedsNoise) {
-    if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, p.t, p.identical_workers ? 0u : threadIdx.x);
+    if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, p.t, p.identical_workers ? 0u : p.worker_base + threadIdx.x);
     __syncthreads();
   }
 
@@ -408,7 +409,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_adagrad(const SweepParams p
   const uint32_t W = (W_ > 0) ? (uint32_t)W_ : p.W;
   __shared__ uint64_t keys[kMaxWorkers];
   if (kNeedsNoise) {
-    if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, p.t, p.identical_workers ? 0u : threadIdx.x);
+    if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, p.t, p.identical_workers ? 0u : p.worker_base + threadIdx.x);
     __syncthreads();
   }
   const float eps2 = __fmul_rn(p.eps, p.eps);

@@ -77,6 +77,16 @@ def lib() -> C.CDLL:
             "la_get_counters": [vp, C.POINTER(u64), C.POINTER(u32), C.POINTER(u64)],
             "la_set_counters": [vp, u64, u32, u64],
             "la_get_stats": [vp, C.POINTER(la_stats), i32],
+            "la_set_worker_range": [vp, u32, u32],
+            "la_comm_create": [vp, u32, u32],
+            "la_comm_buffer": [vp, C.POINTER(vp), C.POINTER(u64)],
+            "la_comm_ipc_handle": [vp, vp],
+            "la_comm_open_peer": [vp, u32, vp],
+            "la_comm_set_peer": [vp, u32, vp],
+            "la_comm_export": [vp],
+            "la_comm_combine": [vp],
+            "la_comm_import": [vp],
+            "la_stream_sync": [vp],
         }
         for name, args in sig.items():
             fn = getattr(L, name)
@@ -284,5 +294,41 @@ class LocalAdaAlter:
         return {k: getattr(st, k) for k, _ in la_stats._fields_}
 
     def sync_stream(self):
-        """Block until the context's stream is idle (uses a zero-length state read)."""
-        self._ck(self.L.la_read_range(self.h, 0, 0, 0, None, None, None))
+        """Block until the context's stream is idle."""
+        self._ck(self.L.la_stream_sync(self.h))
+
+    stream_sync = sync_stream
+
+    # ------------------------------------------------------------------ sharding by worker
+    def set_worker_range(self, worker_base, W_total):
+        self._ck(self.L.la_set_worker_range(self.h, int(worker_base), int(W_total)))
+
+    def comm_create(self, rank, world):
+        self._ck(self.L.la_comm_create(self.h, int(rank), int(world)))
+
+    def comm_buffer(self):
+        """(device pointer, bytes) of the exchange buffer."""
+        p, n = C.c_void_p(), C.c_uint64()
+        self._ck(self.L.la_comm_buffer(self.h, C.byref(p), C.byref(n)))
+        return p.value, n.value
+
+    def comm_ipc_handle(self) -> bytes:
+        buf = C.create_string_buffer(64)
+        self._ck(self.L.la_comm_ipc_handle(self.h, buf))
+        return buf.raw
+
+    def comm_open_peer(self, peer_rank, handle: bytes):
+        buf = C.create_string_buffer(handle, 64)
+        self._ck(self.L.la_comm_open_peer(self.h, int(peer_rank), buf))
+
+    def comm_set_peer(self, peer_rank, dev_ptr):
+        self._ck(self.L.la_comm_set_peer(self.h, int(peer_rank), C.c_void_p(int(dev_ptr))))
+
+    def comm_export(self):
+        self._ck(self.L.la_comm_export(self.h))
+
+    def comm_combine(self):
+        self._ck(self.L.la_comm_combine(self.h))
+
+    def comm_import(self):
+        self._ck(self.L.la_comm_import(self.h))

@@ -1,0 +1,113 @@
+"""Sharding by worker on the GPU: the three-phase synchronisation (export / combine / import)
+against the single-context kernels and the oracle.  One GPU is available, so several ranks are
+emulated as several contexts of one process on one stream (their kernels never wait for each
+other; the host orders the phases)."""
+import numpy as np
+import pytest
+
+from oracle.oracle import Oracle
+from paper_1911_09030_b200 import local_adaalter as la
+from paper_1911_09030_b200.worker_sharded import CudaEngine, WorkerShardedJob
+
+pytestmark = pytest.mark.gpu
+
+
+def _arrays(n, seed):
+    rng = np.random.default_rng(seed)
+    return rng.uniform(0.1, 10, n).astype(np.float32), rng.standard_normal(n).astype(np.float32)
+
+
+def _single(n, W, H, a, c, T):
+    g = la.LocalAdaAlter([n], W, 0.1, 1.0, H)
+    g.set_grad_quadratic(9, a, c, 0.3)
+    g.run(T)
+    return g
+
+
+@pytest.mark.parametrize("n", [64, 1000, 70001])
+def test_world_of_one_equals_la_sync(n):
+    W, H, T = 4, 3, 10
+    a, c = _arrays(n, n)
+    ref = _single(n, W, H, a, c, T)
+    g = la.LocalAdaAlter([n], W, 0.1, 1.0, la.LA_H_NEVER)
+    g.set_grad_quadratic(9, a, c, 0.3)
+    job = WorkerShardedJob(CudaEngine(g, 0, 1), H, exchange="peer")
+    job.run(T)
+    assert g.get_counters() == ref.get_counters() == (T, T % H, T // H)
+    for i in range(W):
+        for u, v in zip(g.read_state(i), ref.read_state(i)):
+            assert np.array_equal(u.view(np.uint32), v.view(np.uint32))
+
+
+@pytest.mark.parametrize("world,W_local", [(2, 4), (4, 2), (2, 1), (3, 2), (8, 2)])
+def test_emulated_ranks_equal_single_gpu_job_bitwise(world, W_local):
+    n, H, T = 5000, 4, 9
+    W_total = world * W_local
+    a, c = _arrays(n, world * 10 + W_local)
+    ref = _single(n, W_total, H, a, c, T)
+    o = Oracle(n, W_total, 0.1, 1.0, H)
+    o.set_grad_quadratic(9, a, c, 0.3)
+    o.run(T)
+    ctxs = []
+    for r in range(world):
+        g = la.LocalAdaAlter([n], W_local, 0.1, 1.0, la.LA_H_NEVER)
+        g.set_grad_quadratic(9, a, c, 0.3)
+        g.comm_create(r, world)
+        ctxs.append(g)
+    for r in range(world):
+        for q in range(world):
+            if q != r:
+                ctxs[r].comm_set_peer(q, ctxs[q].comm_buffer()[0])
+    for t in range(1, T + 1):
+        for g in ctxs:
+            g.local_step()
+        if t % H == 0:
+            for g in ctxs:
+                g.comm_export()
+            for g in ctxs:
+                g.stream_sync()
+            for g in ctxs:
+                g.comm_combine()
+            for g in ctxs:
+                g.stream_sync()
+            for g in ctxs:
+                g.comm_import()
+    for r, g in enumerate(ctxs):
+        assert g.get_counters() == ref.get_counters()
+        for i in range(W_local):
+            gw = r * W_local + i
+            for name, u, v, w in zip("x b2 bs".split(), g.read_state(i), ref.read_state(gw), o.read(gw)):
+                assert np.array_equal(u.view(np.uint32), w.view(np.uint32)), f"{name} vs oracle, rank {r} worker {i}"
+                if W_local & (W_local - 1) == 0:
+                    assert np.array_equal(u.view(np.uint32), v.view(np.uint32)), f"{name} vs single GPU"
+
+
+def test_allreduce_mode_with_one_rank_and_buffer_alias():
+    n, W, H, T = 3000, 8, 2, 6
+    a, c = _arrays(n, 3)
+    ref = _single(n, W, H, a, c, T)
+    g = la.LocalAdaAlter([n], W, 0.1, 1.0, la.LA_H_NEVER)
+    g.set_grad_quadratic(9, a, c, 0.3)
+    eng = CudaEngine(g, 0, 1)
+    job = WorkerShardedJob(eng, H, exchange="allreduce")
+    job.run(T)
+    buf = eng.buffer_tensor()
+    assert buf.is_cuda and buf.numel() == 2 * ((n + 63) // 64 * 64)
+    x0 = g.read_state(0)[0]
+    assert np.array_equal(x0, ref.read_state(0)[0])
+    # after the last import the buffer still holds the totals: mean = total / W
+    np.testing.assert_array_equal((buf[:n].cpu().numpy() / np.float32(W)), x0)
+
+
+def test_misuse_is_reported():
+    g = la.LocalAdaAlter([64], 2, 0.1, 1.0, 2)
+    with pytest.raises(la.LocalAdaAlterError):
+        g.comm_export()                      # no exchange buffer yet
+    g.comm_create(0, 2)
+    with pytest.raises(la.LocalAdaAlterError) as e:
+        g.comm_combine()                     # peer 1 not attached
+    assert "not attached" in str(e.value)
+    with pytest.raises(la.LocalAdaAlterError):
+        g.comm_create(3, 2)
+    with pytest.raises(la.LocalAdaAlterError):
+        g.set_worker_range(7, 8)

@@ -97,3 +97,82 @@ def test_reference_arm_runs_on_rank0_only(tmp_path):
     import json
     doc = json.loads(lines[0])
     assert doc["impl"] == "reference" and doc["cpu_baseline"]["kind"] == "oracle" and doc["value"] > 0
+
+
+WORKER_BY_WORKER = r'''
+import os, sys
+sys.path.insert(0, os.environ["LA_ROOT"])
+import numpy as np, torch, torch.distributed as dist
+from paper_1911_09030_b200.worker_sharded import WorkerShardedJob
+from oracle.oracle import Oracle
+
+class OracleEngine:
+    """CPU stand-in for the CUDA engine (test infrastructure): the local replicas live in an
+    oracle instance; export/import are written out with numpy."""
+    def __init__(self, o, W_local, W_total, n):
+        self.o, self.W, self.W_total, self.n = o, W_local, W_total, n
+        self.buf = torch.zeros(2 * n, dtype=torch.float32)
+    def local_step(self): self.o.local_step()
+    def t_prime(self): return self.o.counters()[1]
+    def stream_sync(self): pass
+    def _tree(self, rows):
+        rows = list(rows)
+        while len(rows) > 1:
+            nxt = [rows[k] + rows[k + 1] for k in range(0, len(rows) - 1, 2)]
+            if len(rows) % 2: nxt.append(rows[-1])
+            rows = nxt
+        return rows[0]
+    def export(self):
+        xs, bs = zip(*[self.o.read(i)[:2] for i in range(self.W)])
+        self.buf[:self.n] = torch.from_numpy(self._tree(xs))
+        self.buf[self.n:] = torch.from_numpy(self._tree(bs))
+    def combine(self): raise AssertionError("peer exchange needs device memory")
+    def buffer_tensor(self): return self.buf
+    def import_(self):
+        w = np.float32(self.W_total)
+        xm = self.buf[:self.n].numpy() / w
+        bm = self.buf[self.n:].numpy() / w
+        for i in range(self.W):
+            self.o.write(i, xm, bm, bm)
+        t, tp, ns = self.o.counters()
+        self.o.set_counters(t, 0, ns + 1)
+
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+n, W_local, H, T = 257, 4, 3, 10
+W_total = W_local * world
+rng = np.random.default_rng(0)
+a = rng.uniform(0.1, 10, n).astype(np.float32); c = rng.standard_normal(n).astype(np.float32)
+o = Oracle(n, W_local, 0.1, 1.0, 0xFFFFFFFF)
+o.set_grad_quadratic(9, a, c, 0.3)
+o.set_worker_base(rank * W_local)
+job = WorkerShardedJob(OracleEngine(o, W_local, W_total, n), H, exchange="allreduce", dist=dist)
+job.run(T)
+mine = np.stack([o.read(i)[0] for i in range(W_local)])
+parts = [None] * world
+dist.all_gather_object(parts, (rank, mine, o.counters(), job.syncs))
+if rank == 0:
+    full = Oracle(n, W_total, 0.1, 1.0, H)
+    full.set_grad_quadratic(9, a, c, 0.3)
+    full.run(T)
+    for r, xs, cnt, syncs in parts:
+        assert cnt == full.counters() and syncs == T // H
+        for i in range(W_local):
+            ref = full.read(r * W_local + i)[0]
+            assert np.array_equal(xs[i].view(np.uint32), ref.view(np.uint32)), (r, i)
+    print("BY_WORKER_OK")
+dist.destroy_process_group()
+'''
+
+
+def test_two_gloo_ranks_sharded_by_worker(tmp_path):
+    """The by-worker choreography (export, all-reduce, import, counters) on two CPU ranks with
+    an oracle-backed engine equals the single-process oracle with W_total workers, bitwise."""
+    script = tmp_path / "by_worker.py"
+    script.write_text(WORKER_BY_WORKER)
+    env = dict(os.environ, LA_ROOT=ROOT, MASTER_ADDR="127.0.0.1")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), str(script)]
+    r = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-4000:]
+    assert "BY_WORKER_OK" in r.stdout
