@@ -43,7 +43,8 @@ enum {
   LA_EINVAL = -1, /* bad argument (NULL handle, N=0, W=0, H=0, eps<=0, non-finite eta, ...) */
   LA_ENOMEM = -2, /* device or host allocation failed, or caller arena too small */
   LA_ECUDA = -3,  /* a CUDA runtime call failed; message in la_last_error */
-  LA_ESTATE = -4  /* call not valid in the context's current configuration */
+  LA_ESTATE = -4, /* call not valid in the context's current configuration */
+  LA_ETOOBIG = -5 /* size exceeds a fixed capacity (la_replica_means_static) */
 };
 
 enum { LA_F32 = 0, LA_BF16 = 1 };               /* gradient dtype */
@@ -200,6 +201,30 @@ int la_comm_combine(la_ctx* ctx);
 int la_comm_import(la_ctx* ctx);
 /* Block until the context's stream is idle. */
 int la_stream_sync(la_ctx* ctx);
+
+/* ---- for callers that must not allocate ------------------------------------------------------
+ * (The paper has no counterpart: this is a deployment variant of the replica average that
+ * la_comm_export / la_comm_import compute.)
+ * Who needs it: programs that gave the whole GPU to their own allocator at start-up and have
+ * nothing left for cudaMalloc (the caller-arena mode of la_create_ex is for them), and services
+ * that ban cudaMalloc/cudaFree once running because both stall the device.  This call makes no
+ * allocation of any kind: its intermediate sums live in a fixed array inside the library image,
+ * 2 * LA_STATIC_SCRATCH_MAX_COORDS floats (8 MiB) on every GPU that loads the library, until
+ * the process exits.
+ *   x_dev, b2_dev    device, [W][stride] floats, 16-byte aligned: the W replicas (read only)
+ *   n, stride        coordinates, and floats between replicas (n <= stride, stride % 4 == 0,
+ *                    stride <= LA_STATIC_SCRATCH_MAX_COORDS, else LA_ETOOBIG)
+ *   x_mean_dev,      device, n floats each: adjacent-pair tree sum over the replicas divided
+ *   b2_mean_dev      by (float)W — the same bits la_sync would put into every replica
+ *   stream           a cudaStream_t (NULL = default); the work is only enqueued
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress) with
+ * that device current; make that first call outside any stream capture.  All calls share the
+ * one array: it is fully rewritten for [0, n) by each call (nothing needs to start at zero, and
+ * it keeps the last call's sums afterwards), so two calls that overlap on the GPU — different
+ * streams, or different threads — race; run them in stream order. */
+#define LA_STATIC_SCRATCH_MAX_COORDS 1048576u
+int la_replica_means_static(const float* x_dev, const float* b2_dev, uint32_t W, uint64_t n, uint64_t stride,
+                            float* x_mean_dev, float* b2_mean_dev, void* stream);
 
 #ifdef __cplusplus
 }

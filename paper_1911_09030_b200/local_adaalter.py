@@ -16,7 +16,8 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "liblocal_adaalter.so")
 
-LA_OK, LA_EINVAL, LA_ENOMEM, LA_ECUDA, LA_ESTATE = 0, -1, -2, -3, -4
+LA_OK, LA_EINVAL, LA_ENOMEM, LA_ECUDA, LA_ESTATE, LA_ETOOBIG = 0, -1, -2, -3, -4, -5
+LA_STATIC_SCRATCH_MAX_COORDS = 1048576
 LA_F32, LA_BF16 = 0, 1
 LA_FUSE_NONE, LA_FUSE_STEP_SYNC, LA_FUSE_SYNC_STEP = 0, 1, 2
 LA_RULE_ADAALTER, LA_RULE_LOCAL_SGD, LA_RULE_ADAGRAD = 0, 1, 2
@@ -87,6 +88,7 @@ def lib() -> C.CDLL:
             "la_comm_combine": [vp],
             "la_comm_import": [vp],
             "la_stream_sync": [vp],
+            "la_replica_means_static": [vp, vp, u32, u64, u64, vp, vp, vp],
         }
         for name, args in sig.items():
             fn = getattr(L, name)
@@ -98,6 +100,14 @@ def lib() -> C.CDLL:
         L.la_last_error.restype = C.c_char_p
         _lib = L
     return _lib
+
+
+def replica_means_static(x_ptr, b2_ptr, W, n, stride, x_mean_ptr, b2_mean_ptr, stream=None) -> int:
+    """`la_replica_means_static`: replica average without any allocation (for callers whose device
+    memory is all spoken for).  Arguments are raw device addresses; returns the status code."""
+    return lib().la_replica_means_static(C.c_void_p(int(x_ptr)), C.c_void_p(int(b2_ptr)), int(W), int(n), int(stride),
+                                         C.c_void_p(int(x_mean_ptr)), C.c_void_p(int(b2_mean_ptr)),
+                                         C.c_void_p(int(stream)) if stream else None)
 
 
 class LocalAdaAlterError(RuntimeError):
