@@ -31,19 +31,17 @@ FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from
 # the ncu capture summarised in profiles/), valid only for the kernel sources they were taken on.
-KERNEL_HASH_AT_CAPTURE = "489667179e4edd72"
-NCU_TRAFFIC_BYTES = {"c2": 2.2238e9}
+KERNEL_HASH_AT_CAPTURE = "bfd46d157b6d8f78"
+NCU_TRAFFIC_BYTES = {"c2": 2.2242e9}
 
 
 def kernel_source_hash():
-    import glob
     import hashlib
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_1911_09030_b200", "csrc")
-    for pat in ("*.cu", "*.cuh", "*.inc"):
-        for f in sorted(glob.glob(os.path.join(d, pat))):
-            with open(f, "rb") as fh:
-                h.update(fh.read())
+    for name in ("grad_source.cuh", "la_sweep.cuh", "la_sweep_inst.inc"):   # the files that define la_sweep
+        with open(os.path.join(d, name), "rb") as fh:
+            h.update(fh.read())
     return h.hexdigest()[:16]
 
 
@@ -280,7 +278,7 @@ def run_ours(args, wl):
             "bound": "hbm", "kernel": "la_sweep<STEP> (K1 local step)", "achieved": achieved, "peak": peak,
             "peak_kind": peak_kind, "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
             "traffic": (NCU_TRAFFIC_BYTES.get(wl.name) if kernel_source_hash() == KERNEL_HASH_AT_CAPTURE
-                        and args.H is None else None),
+                        and args.H is None and args.N is None else None),
             "frac_of_nominal_8TBps": (achieved / NOMINAL_HBM_GBS) if achieved else None,
             "bytes_per_launch": bytes_local, "ms_per_launch": ms_local,
             "bytes_per_update": bytes_local / (wl.W * wl.N),
@@ -415,6 +413,7 @@ def main():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--H", type=int, default=None, help="override the synchronisation period")
     ap.add_argument("--T", type=int, default=None, help="override iterations per step")
+    ap.add_argument("--N", type=int, default=None, help="override the size (one flat tensor), e.g. for small ncu captures")
     ap.add_argument("--fusion", type=int, default=1, help="0 unfused, 1 step+sync, 2 sync+next step")
     ap.add_argument("--blocks-per-sm", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -431,6 +430,8 @@ def main():
         wl.H = args.H
     if args.T is not None:
         wl.T = args.T
+    if args.N is not None:
+        wl.sizes = [args.N]
     if args.impl == "reference":
         run_reference(args, wl)
     else:
