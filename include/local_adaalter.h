@@ -49,7 +49,10 @@ enum {
 
 enum { LA_F32 = 0, LA_BF16 = 1 };               /* gradient dtype */
 enum { LA_FUSE_NONE = 0, LA_FUSE_STEP_SYNC = 1, /* la_run: step t'=H and its sync in one pass */
-       LA_FUSE_SYNC_STEP = 2 };                 /* la_run: sync folded into the following step */
+       LA_FUSE_SYNC_STEP = 2,                   /* la_run: sync folded into the following step */
+       LA_FUSE_PERIOD = 3 };                    /* la_run: up to 8 consecutive local steps (and the sync
+                                                   that closes the period) in one pass over HBM; for the
+                                                   generated gradients, whose noise lives in registers */
 enum { LA_RULE_ADAALTER = 0,  /* Algorithm 3, Local AdaAlter (default) */
        LA_RULE_LOCAL_SGD = 1, /* Algorithm 2: y = x - eta G, x averaged every H steps, no accumulator */
        LA_RULE_ADAGRAD = 2 }; /* Algorithm 1: gradients averaged every step, B^2 += G o G, updated B^2 divides */

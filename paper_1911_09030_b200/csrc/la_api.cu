@@ -13,6 +13,7 @@
 
 #include "../../include/local_adaalter.h"
 #include "la_exchange.cuh"
+#include "la_period.cuh"
 #include "la_sweep.cuh"
 
 namespace la {
@@ -32,6 +33,24 @@ SweepKernel lookup_sweep(int W, int rule, int gm, bool bf16, bool pre, bool step
     case 8: return lookup_sweep_w8(rule, gm, bf16, pre, step, post);
     case 16: return lookup_sweep_w16(rule, gm, bf16, pre, step, post);
     default: return lookup_sweep_w0(rule, gm, bf16, pre, step, post);
+  }
+}
+
+PeriodKernel lookup_period_w0(int, bool, bool);
+PeriodKernel lookup_period_w1(int, bool, bool);
+PeriodKernel lookup_period_w2(int, bool, bool);
+PeriodKernel lookup_period_w4(int, bool, bool);
+PeriodKernel lookup_period_w8(int, bool, bool);
+PeriodKernel lookup_period_w16(int, bool, bool);
+
+PeriodKernel lookup_period(int W, int gm, bool bf16, bool post) {
+  switch (W) {
+    case 1: return lookup_period_w1(gm, bf16, post);
+    case 2: return lookup_period_w2(gm, bf16, post);
+    case 4: return lookup_period_w4(gm, bf16, post);
+    case 8: return lookup_period_w8(gm, bf16, post);
+    case 16: return lookup_period_w16(gm, bf16, post);
+    default: return lookup_period_w0(gm, bf16, post);
   }
 }
 
@@ -291,6 +310,44 @@ int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t
   return LA_OK;
 }
 
+// h consecutive local steps (and, if `post`, the synchronisation that closes the period) in one pass.
+int launch_period(la_ctx* c, uint32_t h, bool post) {
+  const la::PeriodKernel k =
+      la::lookup_period((int)c->W, c->grad_kind, c->bf16 && c->grad_kind <= la::kGradQuadratic, post);
+  if (!k.fn) return fail(c, LA_ESTATE, "no period kernel for this combination (W=%u grad=%d)", c->W, c->grad_kind);
+  la::PeriodParams pp{};
+  la::SweepParams& p = pp.base;
+  p.X = c->X; p.B2 = c->B2; p.Bs = c->Bs;
+  p.a = c->pa; p.c = c->pc; p.s = c->has_s ? c->ps : nullptr;
+  p.n = c->N; p.stride = c->stride; p.j_base = c->j_base;
+  p.seed = c->seed; p.t = c->t; p.W = c->W; p.tp = c->tp;
+  p.warm_up_steps = c->warm_up_steps; p.identical_workers = c->identical ? 1u : 0u;
+  p.worker_base = c->worker_base;
+  p.eta = c->eta; p.eps = c->eps; p.sigma = c->sigma;
+  pp.h = h;
+  const unsigned block = la::kBlockThreads;
+  const uint64_t ngroups = (c->N + (uint64_t)k.vec - 1) / (uint64_t)k.vec;
+  uint64_t blocks = (ngroups + block - 1) / block;
+  // issue-bound kernel: measured optimum around 192 blocks per SM in the grid (sweep 12..4096)
+  const int bps = c->blocks_per_sm > 0 ? c->blocks_per_sm : 192;
+  const uint64_t cap = (uint64_t)c->num_sms * (uint64_t)bps;
+  if (blocks > cap) blocks = cap;
+  EventPair ep{};
+  if (c->profiling) {
+    int rc = begin_timed(c, kClassFused, &ep);
+    if (rc) return rc;
+  }
+  k.fn<<<(unsigned)blocks, block, 0, c->stream>>>(pp);
+  LA_CUDA(c, cudaGetLastError());
+  if (c->profiling) {
+    LA_CUDA(c, cudaEventRecord(ep.b, c->stream));
+    c->pending.push_back(ep);
+  }
+  c->stats.launches_fused++;
+  c->stats.bytes_fused += pass_bytes(c, false, true, post, c->grad_kind);
+  return LA_OK;
+}
+
 int upload_padded(la_ctx* c, float* dst, const float* src_host, float pad) {
   // dst has `stride` floats; [0,N) from the host, the tail [N,stride) = pad.
   LA_CUDA(c, cudaMemcpyAsync(dst, src_host, c->N * sizeof(float), cudaMemcpyHostToDevice, c->stream));
@@ -480,7 +537,7 @@ int la_set_warmup(la_ctx* c, uint32_t steps) {
 
 int la_set_fusion(la_ctx* c, int mode) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
-  if (mode != LA_FUSE_NONE && mode != LA_FUSE_STEP_SYNC && mode != LA_FUSE_SYNC_STEP)
+  if (mode != LA_FUSE_NONE && mode != LA_FUSE_STEP_SYNC && mode != LA_FUSE_SYNC_STEP && mode != LA_FUSE_PERIOD)
     return fail(c, LA_EINVAL, "unknown fusion mode %d", mode);
   c->fusion = mode;
   return LA_OK;
@@ -557,7 +614,30 @@ int la_run(la_ctx* c, uint64_t T) {
     }
     return LA_OK;
   }
+  if (c->fusion == LA_FUSE_PERIOD && c->rule == LA_RULE_ADAALTER) {
+    // temporal blocking: up to kPeriodMax local steps per pass, the closing one with its sync
+    uint64_t left = T;
+    while (left > 0) {
+      if (c->tp >= c->H) {  // only after manual stepping past H: behave like the plain loop
+        int rc = la_local_step(c);
+        if (rc) return rc;
+        left -= 1;
+        continue;
+      }
+      uint64_t h = (uint64_t)(c->H - c->tp);
+      if (h > left) h = left;
+      if (h > (uint64_t)la::kPeriodMax) h = la::kPeriodMax;
+      const bool closes = (c->tp + h == c->H);
+      int rc = launch_period(c, (uint32_t)h, closes);
+      if (rc) return rc;
+      c->t += h;
+      if (closes) { c->tp = 0; c->nsync += 1; } else { c->tp += (uint32_t)h; }
+      left -= h;
+    }
+    return LA_OK;
+  }
   bool deferred = false;
+  const int fusion = (c->fusion == LA_FUSE_PERIOD) ? LA_FUSE_STEP_SYNC : c->fusion;  // baselines: step+sync
   for (uint64_t k = 0; k < T; ++k) {
     int rc;
     if (deferred) {
@@ -565,7 +645,7 @@ int la_run(la_ctx* c, uint64_t T) {
       if (rc) return rc;
       c->nsync += 1; c->t += 1; c->tp = 1;
       deferred = false;
-    } else if (c->fusion == LA_FUSE_STEP_SYNC && c->tp + 1 == c->H) {
+    } else if (fusion == LA_FUSE_STEP_SYNC && c->tp + 1 == c->H) {
       rc = launch_sweep(c, false, true, true, c->t + 1, c->tp + 1, c->grad_kind, nullptr);  // K3: step t'=H and its sync
       if (rc) return rc;
       c->t += 1; c->tp = 0; c->nsync += 1;
@@ -575,7 +655,7 @@ int la_run(la_ctx* c, uint64_t T) {
       if (rc) return rc;
     }
     if (c->tp == c->H) {
-      if (c->fusion == LA_FUSE_SYNC_STEP && k + 1 < T) {
+      if (fusion == LA_FUSE_SYNC_STEP && k + 1 < T) {
         deferred = true;
       } else {
         rc = la_sync(c);  // K2

@@ -79,11 +79,15 @@ def test_config2_flat_scaled_noise():
     _run_config("c2", span=1024, extra=2)
 
 
+def test_config2_period_fusion():
+    _run_config("c2", fusion=la.LA_FUSE_PERIOD, span=1024, extra=2)
+
+
 def test_config3_six_tensors_quadratic():
     _run_config("c3", span=2048, extra=3)
 
 
-@pytest.mark.parametrize("H,fusion", [(1, 2), (4, 0), (16, 1), (64, 2)])
+@pytest.mark.parametrize("H,fusion", [(1, 2), (4, 0), (16, 1), (64, 2), (16, 3)])
 def test_config4_sync_period_sweep(H, fusion):
     _run_config("c4", H=H, fusion=fusion, span=512, extra=2)
 
@@ -92,3 +96,4 @@ def test_config5_ragged_bf16():
     wl = workloads.config("c5")
     assert len(wl.sizes) == 200 and min(wl.sizes) >= 1024 and abs(wl.N - 4e8) < 4e6
     _run_config("c5", span=1024, extra=2)
+    _run_config("c5", fusion=la.LA_FUSE_PERIOD, span=512, extra=1)

@@ -25,7 +25,7 @@ def _arrays(n, seed):
 
 
 # ----------------------------------------------------------------------------- configuration 1
-@pytest.mark.parametrize("fusion", [0, 1, 2])
+@pytest.mark.parametrize("fusion", [0, 1, 2, 3])
 def test_config1_full(fusion):
     wl = workloads.config("c1")
     arr = wl.arrays()
@@ -47,7 +47,7 @@ def test_tails_and_worker_counts(n, W):
     T = 7
     arr = _arrays(n, 10 * n + W)
     for H, grad, fusion in [(1, "quadratic", 0), (2, "noise_scaled", 1), (3, "quadratic", 2), (T, "noise", 1),
-                            (T + 1, "quadratic", 2)]:
+                            (T + 1, "quadratic", 2), (3, "quadratic", 3), (T + 1, "noise_scaled", 3)]:
         g, o = make_pair(n, W, 0.1, 0.5, H, grad, seed=n + W, arrays=arr, sigma=0.3, fusion=fusion, b0sq=0.25)
         g.run(T)
         o.run(T)
@@ -59,7 +59,7 @@ def test_tails_and_worker_counts(n, W):
 def test_generic_worker_counts(W):
     n, T = 257, 9
     arr = _arrays(n, W)
-    for H, fusion in [(2, 0), (3, 1), (4, 2)]:
+    for H, fusion in [(2, 0), (3, 1), (4, 2), (4, 3)]:
         g, o = make_pair(n, W, 0.05, 1.0, H, "quadratic", seed=W, arrays=arr, sigma=1.0, fusion=fusion)
         g.run(T)
         o.run(T)
@@ -69,7 +69,7 @@ def test_generic_worker_counts(W):
 @pytest.mark.parametrize("grad,bf16", [("noise", False), ("noise", True), ("noise_scaled", False),
                                        ("noise_scaled", True), ("quadratic", False), ("quadratic", True),
                                        ("constant", False)])
-@pytest.mark.parametrize("fusion", [0, 1, 2])
+@pytest.mark.parametrize("fusion", [0, 1, 2, 3])
 def test_gradient_modes(grad, bf16, fusion):
     n, W, H, T = 70001, 4, 3, 10      # several blocks and a ragged tail
     arr = _arrays(n, 3)
@@ -88,7 +88,7 @@ def test_fused_kernels_equal_unfused_bitwise(W, H):
     n, T = 12345, 11
     arr = _arrays(n, 77)
     states = []
-    for fusion in (0, 1, 2):
+    for fusion in (0, 1, 2, 3):
         g = la.LocalAdaAlter([n], W, 0.1, 1.0, H)
         g.set_grad_quadratic(5, arr["a"], arr["c"], 0.2)
         g.set_fusion(fusion)
@@ -104,11 +104,14 @@ def test_fused_kernels_equal_unfused_bitwise(W, H):
     assert states[0][2]["launches_fused"] == 0 and states[0][2]["launches_sync"] == T // H
     assert states[1][2]["launches_fused"] == T // H and states[1][2]["launches_sync"] == 0
     assert states[2][2]["launches_fused"] > 0
+    # temporal blocking: one pass per (piece of a) period, nothing else
+    assert states[3][2]["launches_local"] == 0 and states[3][2]["launches_sync"] == 0
+    assert states[3][2]["launches_fused"] <= -(-4 // min(H, 8)) + -(-(T - 4) // min(H, 8)) + 2
 
 
 # ----------------------------------------------------------------------------- schedule
 @pytest.mark.parametrize("H,T", [(1, 5), (2, 5), (3, 9), (5, 5), (6, 5), (la.LA_H_NEVER, 6)])
-@pytest.mark.parametrize("fusion", [0, 1, 2])
+@pytest.mark.parametrize("fusion", [0, 1, 2, 3])
 def test_schedule_counters_match_oracle(H, T, fusion):
     g, o = make_pair(64, 2, 0.1, 1.0, H, "noise", seed=1, fusion=fusion)
     for _ in range(T):
@@ -130,10 +133,22 @@ def test_manual_steps_and_sync():
     assert g.get_counters() == (4, 0, 3)
 
 
-def test_warmup_matches_oracle():
-    g, o = make_pair(513, 4, 0.5, 1.0, 4, "noise", seed=8, warmup=6, b0sq=1.0)
+@pytest.mark.parametrize("fusion", [1, 3])
+def test_warmup_matches_oracle(fusion):
+    g, o = make_pair(513, 4, 0.5, 1.0, 4, "noise", seed=8, warmup=6, b0sq=1.0, fusion=fusion)
     g.run(11); o.run(11)
     compare(g, o, 4, TOL_RUN)
+
+
+@pytest.mark.parametrize("H,T,W", [(20, 50, 4), (8, 64, 8), (64, 70, 16), (5, 23, 2), (9, 9, 3)])
+def test_period_fusion_long_periods(H, T, W):
+    """Periods longer than one pass (8 steps) are cut into pieces; run boundaries fall anywhere."""
+    n = 3001
+    arr = _arrays(n, H)
+    g, o = make_pair(n, W, 0.05, 0.5, H, "quadratic", seed=H, arrays=arr, sigma=0.4, fusion=3)
+    g.run(3); g.run(T - 3)
+    o.run(T)
+    compare(g, o, W, TOL_RUN)
 
 
 def test_initial_iterate_and_b0():
