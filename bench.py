@@ -31,17 +31,22 @@ FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from
 # the ncu capture summarised in profiles/), valid only for the kernel sources they were taken on.
-KERNEL_HASH_AT_CAPTURE = "bfd46d157b6d8f78"
+KERNEL_HASH_AT_CAPTURE = "629bbcd81a8733ae"
 NCU_TRAFFIC_BYTES = {"c2": 2.2242e9}
 
 
 def kernel_source_hash():
+    """Hash of what defines the la_sweep kernels: the two headers and the tuning macros."""
     import hashlib
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_1911_09030_b200", "csrc")
-    for name in ("grad_source.cuh", "la_sweep.cuh", "la_sweep_inst.inc"):   # the files that define la_sweep
+    for name in ("grad_source.cuh", "la_sweep.cuh"):
         with open(os.path.join(d, name), "rb") as fh:
             h.update(fh.read())
+    with open(os.path.join(d, "la_sweep_inst.inc")) as fh:
+        for line in fh:
+            if line.startswith("#define LA_VEC") or line.startswith("#define LA_MINB"):
+                h.update(line.encode())
     return h.hexdigest()[:16]
 
 
@@ -164,6 +169,27 @@ def run_reference(args, wl):
     print(json.dumps(line), flush=True)
 
 
+# Issue-slot roofline of the temporal-blocking kernel (la_period): 148 SMs x 4 schedulers x 32
+# lanes = 18 944 lane-instructions per clock; lane-instructions per worker*param update from the
+# ncu capture summarised in profiles/ (smsp__inst_executed.sum x 32 / updates per launch).
+LANE_INSTR_PER_CLOCK = 148 * 4 * 32
+PERIOD_LANE_INSTR_PER_UPDATE = {"c2": 49.8}
+
+
+def alu_roofline(period, wl, clocks):
+    if period is None:
+        return None
+    out = dict(period)
+    ipu = PERIOD_LANE_INSTR_PER_UPDATE.get(wl.name)
+    max_mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+    peak = LANE_INSTR_PER_CLOCK * max_mhz * 1e6 / 1e12          # T lane-instr/s at the maximum SM clock
+    if ipu:
+        ach = period["value"] * ipu / 1e12
+        out["roofline"] = {"bound": "alu", "achieved": ach, "peak": peak, "unit": "T lane-instr/s",
+                           "frac": ach / peak, "lane_instr_per_update": ipu, "traffic": None}
+    return out
+
+
 def workload_config(wl, args):
     return {"workload": f"{wl.name}: W={wl.W}, N={wl.N} fp32 in {len(wl.sizes)} tensor(s), grad={wl.grad}"
                         f"{'+bf16' if wl.bf16_grads else ''}, eta={wl.eta}, eps={wl.eps}, H={wl.H}, T={wl.T} per step",
@@ -246,6 +272,27 @@ def run_ours(args, wl):
     ctx.set_profiling(False)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
 
+    # ---- the same job with temporal blocking (LA_FUSE_PERIOD): issue-bound instead of HBM-bound
+    period = None
+    if args.fusion != la.LA_FUSE_PERIOD and not args.no_period:
+        ctx.set_fusion(la.LA_FUSE_PERIOD)
+        for _ in range(2):
+            ctx.run(wl.T)
+        barrier()
+        ctx.get_stats(reset=True)
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record(stream)
+        for _ in range(args.steps):
+            ctx.run(wl.T)
+        p1.record(stream)
+        barrier()
+        pst = ctx.get_stats(reset=True)
+        pms = sharding.max_over_ranks(p0.elapsed_time(p1) / args.steps, dist if world > 1 else None)
+        period = {"ms_per_step": pms, "value": wl.W * wl.N * wl.T * world / (pms * 1e-3), "unit": UNIT,
+                  "launches_per_step": pst["launches_fused"] // args.steps,
+                  "hbm_GBps": pst["bytes_fused"] / args.steps / (pms * 1e-3) / 1e9}
+        ctx.set_fusion(args.fusion)
+
     # ---- end to end through the C-ABI with host buffers -------------------------------------
     def e2e_step():
         upload()
@@ -309,6 +356,7 @@ def run_ours(args, wl):
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": int(sum(launches.values())),
             "roofline": roofline, "cpu_baseline": cpu, "kernels": per_class,
+            "temporal_blocking": alu_roofline(period, wl, clocks),
             "hbm_GBps_whole_step": (stats["bytes_local"] + stats["bytes_sync"] + stats["bytes_fused"]) / (ms_total * 1e-3) / 1e9,
         }
         print(json.dumps(line), flush=True)
@@ -417,6 +465,7 @@ def main():
     ap.add_argument("--fusion", type=int, default=1, help="0 unfused, 1 step+sync, 2 sync+next step")
     ap.add_argument("--blocks-per-sm", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-period", action="store_true", help="skip the extra temporal-blocking measurement")
     ap.add_argument("--report", action="store_true", help="all configurations + the H sweep (not the JSON line)")
     ap.add_argument("--report-out", default=None)
     args = ap.parse_args()
