@@ -142,6 +142,11 @@ int la_local_step(la_ctx* ctx);
  * dtype LA_F32 (4 bytes) or LA_BF16 (2 bytes, widened exactly).  16-byte aligned. Not retained
  * beyond the kernel; the caller must keep it alive until the stream reaches that point. */
 int la_local_step_grads(la_ctx* ctx, const void* g_dev, int dtype);
+/* One COMPLETE iteration of Algorithm 3 with caller-supplied gradients (same table as above):
+ * the local step and, when it makes t' reach H, the synchronisation branch — in the same pass
+ * over memory unless the fusion mode is LA_FUSE_NONE.  This is the call a trainer makes once per
+ * optimizer step after back-propagation. */
+int la_step_grads(la_ctx* ctx, const void* g_dev, int dtype);
 /* Synchronisation branch of Algorithm 3: x and B^2 of every worker are replaced by the means
  * over workers; the mean B^2 becomes the stale denominator; t' = 0; n_sync += 1.  Legal at any
  * time (outside la_run it need not fall on a multiple of H). */

@@ -276,6 +276,10 @@ int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t
   p.X = c->X; p.B2 = c->B2; p.Bs = c->Bs;
   p.a = c->pa; p.c = c->pc; p.s = c->has_s ? c->ps : nullptr;
   p.gext = gext;
+  if (gext) {
+    const uint64_t elem = (gm == la::kGradExternalBF16) ? 2 : 4;
+    p.gext_vec = (c->N % (uint64_t)k.vec == 0 && (reinterpret_cast<uintptr_t>(gext) % ((uint64_t)k.vec * elem)) == 0) ? 1u : 0u;
+  }
   p.n = c->N; p.stride = c->stride; p.j_base = c->j_base;
   p.seed = c->seed; p.t = t; p.W = c->W; p.tp = tp;
   p.warm_up_steps = c->warm_up_steps; p.identical_workers = c->identical ? 1u : 0u;
@@ -589,6 +593,27 @@ int la_local_step_grads(la_ctx* c, const void* g_dev, int dtype) {
                         dtype == LA_F32 ? la::kGradExternalF32 : la::kGradExternalBF16, g_dev);
   if (rc) return rc;
   c->t += 1; c->tp += 1;
+  return LA_OK;
+}
+
+int la_step_grads(la_ctx* c, const void* g_dev, int dtype) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!g_dev) return fail(c, LA_EINVAL, "g_dev is NULL");
+  if (dtype != LA_F32 && dtype != LA_BF16) return fail(c, LA_EINVAL, "dtype must be LA_F32 or LA_BF16");
+  if (c->rule != LA_RULE_ADAALTER) return fail(c, LA_ESTATE, "supplied gradients are implemented for Local AdaAlter only");
+  DeviceGuard guard(c->device);
+  const int gm = dtype == LA_F32 ? la::kGradExternalF32 : la::kGradExternalBF16;
+  const bool closes = (c->tp + 1 == c->H);
+  if (closes && c->fusion != LA_FUSE_NONE) {
+    int rc = launch_sweep(c, false, true, true, c->t + 1, c->tp + 1, gm, g_dev);  // step and its sync in one pass
+    if (rc) return rc;
+    c->t += 1; c->tp = 0; c->nsync += 1;
+    return LA_OK;
+  }
+  int rc = launch_sweep(c, false, true, false, c->t + 1, c->tp + 1, gm, g_dev);
+  if (rc) return rc;
+  c->t += 1; c->tp += 1;
+  if (c->tp == c->H) return la_sync(c);
   return LA_OK;
 }
 

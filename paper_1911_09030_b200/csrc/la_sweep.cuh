@@ -40,6 +40,7 @@ struct SweepParams {
   const float* c;  // [stride] or null
   const float* s;  // [stride] or null
   const void* gext;    // external gradients, [W][N]
+  uint32_t gext_vec;   // 1: every row of gext is aligned for V-wide loads (N % V == 0, aligned base)
   uint64_t n;          // logical coordinates N
   uint64_t stride;     // replica stride in floats (multiple of 64, >= N rounded up to 4)
   uint64_t j_base;     // global index of coordinate 0 (multiple of 4)
@@ -214,6 +215,56 @@ __device__ __forceinline__ void store_replica(uint64_t& addr, uint64_t b_delta, 
   advance(addr, stride_bytes);
 }
 
+// Caller-supplied gradients of CH consecutive replicas for one coordinate group (fp32 or bf16
+// table [W][N], worker-major), fetched together with the replicas so that they are in flight
+// while the previous chunk is consumed.
+template <int V, int CH>
+struct GradChunk {
+  Vec<V> g[CH];
+};
+
+template <int GM, int V, int CH>
+__device__ __forceinline__ void load_grads(GradChunk<V, CH>& gc, const SweepParams& p, uint64_t& g_addr,
+                                           uint64_t row_bytes, uint32_t W, uint32_t i0, uint64_t off) {
+  constexpr bool kF32 = (GM == kGradExternalF32);
+#pragma unroll
+  for (int k = 0; k < CH; ++k)
+    if (i0 + k < W) {
+      if (p.gext_vec) {
+        if (kF32) {
+          gc.g[k] = ld_stream<V>(as_ptr(g_addr));
+        } else {
+          // V bf16 values in one 32- or 64-bit load; widening bf16 -> fp32 is exact
+          if (V == 2) {
+            const uint32_t w = __ldcs(reinterpret_cast<const uint32_t*>(g_addr));
+            gc.g[k].v[0] = __uint_as_float(w << 16);
+            gc.g[k].v[1] = __uint_as_float(w & 0xFFFF0000u);
+          } else {
+            const uint2 w = __ldcs(reinterpret_cast<const uint2*>(g_addr));
+            gc.g[k].v[0] = __uint_as_float(w.x << 16);
+            gc.g[k].v[1] = __uint_as_float(w.x & 0xFFFF0000u);
+            gc.g[k].v[V - 2] = __uint_as_float(w.y << 16);
+            gc.g[k].v[V - 1] = __uint_as_float(w.y & 0xFFFF0000u);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+          float v = 0.0f;
+          if (off + e < p.n) {
+            if (kF32) {
+              v = __ldcs(reinterpret_cast<const float*>(g_addr) + e);
+            } else {
+              v = __uint_as_float((uint32_t)__ldcs(reinterpret_cast<const unsigned short*>(g_addr) + e) << 16);
+            }
+          }
+          gc.g[k].v[e] = v;
+        }
+      }
+      advance(g_addr, row_bytes);
+    }
+}
+
 // r = eta_t / sqrt(B^2_{t-t'} + t' eps^2): the step size all workers share (Section 4.2).
 template <int V>
 __device__ __forceinline__ Vec<V> step_size(const Vec<V>& bs, float q, float eta_t) {
@@ -232,21 +283,6 @@ __device__ __forceinline__ Vec<V> gradient(const SweepParams& p, const CoordInpu
   Vec<V> g;
   if (GM == kGradConstant) {
     return in.s;
-  } else if (GM == kGradExternalF32 || GM == kGradExternalBF16) {
-    const uint64_t base = (uint64_t)worker * p.n + off;
-#pragma unroll
-    for (int k = 0; k < V; ++k) {
-      g.v[k] = 0.0f;
-      if (off + k < p.n) {
-        if (GM == kGradExternalF32) {
-          g.v[k] = __ldcs(reinterpret_cast<const float*>(p.gext) + base + k);
-        } else {
-          const unsigned short h = __ldcs(reinterpret_cast<const unsigned short*>(p.gext) + base + k);
-          g.v[k] = __uint_as_float((uint32_t)h << 16);  // bf16 -> fp32 is exact
-        }
-      }
-    }
-    return g;
   } else {
     Vec<V> xi;
 #pragma unroll
@@ -320,11 +356,19 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
   const uint64_t b_delta = reinterpret_cast<uint64_t>(p.B2) - x_base;
   const uint64_t stride_bytes = p.stride * sizeof(float);
 
+  constexpr bool kExternal = STEP && (GM == kGradExternalF32 || GM == kGradExternalBF16);
+  constexpr uint64_t kGradElem = (GM == kGradExternalBF16) ? 2 : 4;
+  const uint64_t g_base = reinterpret_cast<uint64_t>(p.gext);
+  const uint64_t g_row_bytes = p.n * kGradElem;
+
   ReplicaChunk<V, CH> nxt;
+  GradChunk<V, kExternal ? CH : 1> gnxt;
   CoordInputs<V> in_next;
   load_coord<GM, STEP, kLoadsBs, V>(in_next, p, grp * V);
   uint64_t ld_addr = x_base + grp * (V * sizeof(float));
+  uint64_t g_addr = g_base + grp * (V * kGradElem);
   load_chunk<V, CH, ACC>(nxt, ld_addr, b_delta, stride_bytes, W, 0u);
+  if (kExternal) load_grads<GM, V, kExternal ? CH : 1>(gnxt, p, g_addr, g_row_bytes, W, 0u, grp * V);
 
   for (;;) {
     const uint64_t off = grp * V;
@@ -342,12 +386,18 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
 #pragma unroll kOuterUnroll
     for (uint32_t i0 = 0; i0 < W; i0 += CH) {
       ReplicaChunk<V, CH> cur = nxt;
+      GradChunk<V, kExternal ? CH : 1> gcur = gnxt;
       if (i0 + CH < W) {
         load_chunk<V, CH, ACC>(nxt, ld_addr, b_delta, stride_bytes, W, i0 + CH);
+        if (kExternal) load_grads<GM, V, kExternal ? CH : 1>(gnxt, p, g_addr, g_row_bytes, W, i0 + CH, off);
       } else if (has_next) {
         load_coord<GM, STEP, kLoadsBs, V>(in_next, p, next_grp * V);
         ld_addr = x_base + next_grp * (V * sizeof(float));
         load_chunk<V, CH, ACC>(nxt, ld_addr, b_delta, stride_bytes, W, 0u);
+        if (kExternal) {
+          g_addr = g_base + next_grp * (V * kGradElem);
+          load_grads<GM, V, kExternal ? CH : 1>(gnxt, p, g_addr, g_row_bytes, W, 0u, next_grp * V);
+        }
       }
       asm volatile("" ::: "memory");
 #pragma unroll
@@ -357,7 +407,8 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
           if (PRE) {
             tree.push(i, cur.x[k], cur.b[k]);
           } else {
-            const Vec<V> g = gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
+            const Vec<V> g = kExternal ? gcur.g[kExternal ? k : 0]
+                                       : gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
             apply<V, ACC>(r, g, cur.x[k], cur.b[k]);
             if (POST) {
               tree.push(i, cur.x[k], cur.b[k]);

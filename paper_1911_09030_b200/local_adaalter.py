@@ -69,6 +69,7 @@ def lib() -> C.CDLL:
             "la_set_profiling": [vp, i32],
             "la_local_step": [vp],
             "la_local_step_grads": [vp, vp, i32],
+            "la_step_grads": [vp, vp, i32],
             "la_sync": [vp],
             "la_run": [vp, u64],
             "la_read_state": [vp, u32, vp, vp, vp],
@@ -255,6 +256,9 @@ class LocalAdaAlter:
 
     def local_step_grads(self, g_dev_ptr: int, dtype=LA_F32):
         self._ck(self.L.la_local_step_grads(self.h, C.c_void_p(int(g_dev_ptr)), int(dtype)))
+
+    def step_grads(self, g_dev_ptr: int, dtype=LA_F32):
+        self._ck(self.L.la_step_grads(self.h, C.c_void_p(int(g_dev_ptr)), int(dtype)))
 
     def sync(self):
         self._ck(self.L.la_sync(self.h))

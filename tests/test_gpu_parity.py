@@ -238,6 +238,40 @@ def test_supplied_gradients_match_oracle(dtype, n):
     compare(g, o, W, TOL_RUN)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("W,n,H,fusion", [(4, 70002, 3, 1), (8, 4098, 2, 0), (16, 1000, 4, 1), (3, 777, 2, 1),
+                                           (2, 12, 1, 1), (5, 4100, 3, 2)])
+def test_step_grads_full_iteration(dtype, W, n, H, fusion):
+    """la_step_grads = local step + the synchronisation when it is due (fused or not); even n takes
+    the vector loads, odd n the scalar ones; a table offset by one element is mis-aligned."""
+    import torch
+    T = 7
+    rng = np.random.default_rng(n + W)
+    g = la.LocalAdaAlter([n], W, 0.3, 0.5, H, b0sq=0.25)
+    g.set_init(None, 0.25)
+    g.set_fusion(fusion)
+    o = Oracle(n, W, 0.3, 0.5, H, 0.25)
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    code = la.LA_F32 if dtype == "f32" else la.LA_BF16
+    for t in range(T):
+        G = torch.from_numpy(rng.standard_normal((W, n)).astype(np.float32)).to(tdt)
+        pad = 1 if t == 2 else 0                                   # once: a mis-aligned table
+        buf = torch.empty(W * n + pad, dtype=tdt, device="cuda")
+        buf[pad:] = G.reshape(-1).cuda()
+        g.step_grads(buf[pad:].data_ptr(), code)
+        o.local_step(G.float().numpy())
+        if o.counters()[1] == H:
+            o.sync()
+        g.sync_stream()
+        assert g.get_counters() == o.counters()
+    compare(g, o, W, TOL_RUN)
+    st = g.get_stats()
+    if fusion == 0:
+        assert st["launches_fused"] == 0 and st["launches_sync"] == T // H
+    else:
+        assert st["launches_fused"] == T // H and st["launches_sync"] == 0
+
+
 def test_checkpoint_resume_bitwise():
     n, W, H = 3001, 4, 4
     arr = _arrays(n, 6)
