@@ -97,3 +97,26 @@ def test_config5_ragged_bf16():
     assert len(wl.sizes) == 200 and min(wl.sizes) >= 1024 and abs(wl.N - 4e8) < 4e6
     _run_config("c5", span=1024, extra=2)
     _run_config("c5", fusion=la.LA_FUSE_PERIOD, span=512, extra=1)
+
+
+def test_beyond_32_bit_indexing():
+    """W x N above 2^32 elements (17 GiB per state array): every offset computation is 64-bit.
+    Checked on windows at both ends of the vector and around the 2^32-byte and 2^32-element
+    marks of replica rows."""
+    N, W, H, T = (1 << 30) + 6, 4, 3, 4
+    g = la.LocalAdaAlter.with_torch_arena([N], W, 0.05, 0.5, H, b0sq=0.0)
+    g.set_grad_noise(11, None)
+    g.set_fusion(la.LA_FUSE_STEP_SYNC)
+    g.run(2)
+    g.set_fusion(la.LA_FUSE_PERIOD)
+    g.run(T - 2)
+    ranges = [(0, 256), ((1 << 29) - 128, (1 << 29) + 128), (N - 262, N), (123456788, 123456788 + 200)]
+    for lo, hi in ranges:
+        o = Oracle(hi - lo, W, 0.05, 0.5, H, 0.0, j_base=lo)
+        o.set_grad_noise(11, None)
+        o.run(T)
+        for i in range(W):
+            for a, b in zip(g.read_range(i, lo, hi - lo), o.read(i)):
+                assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), (lo, i)
+        assert g.get_counters() == o.counters()
+    g.close()

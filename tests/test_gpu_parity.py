@@ -121,6 +121,17 @@ def test_schedule_counters_match_oracle(H, T, fusion):
     compare(g, o, 2, TOL_RUN)
 
 
+def test_zero_length_run_and_repeated_sync_are_harmless():
+    g, o = make_pair(33, 4, 0.2, 1.0, 2, "noise", seed=3)
+    g.run(0); o.run(0)
+    assert g.get_counters() == (0, 0, 0)
+    g.sync(); o.sync()                      # averaging identical replicas: the identity
+    x, b2, bs = g.read_state(3)
+    assert np.all(x == 0) and np.all(b2 == 0) and np.all(bs == 0)
+    g.run(5); o.run(5)
+    compare(g, o, 4, TOL_RUN)
+
+
 def test_manual_steps_and_sync():
     g, o = make_pair(100, 4, 0.2, 1.0, 10, "noise", seed=3)
     for k in range(3):
