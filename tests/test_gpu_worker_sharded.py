@@ -111,3 +111,61 @@ def test_misuse_is_reported():
         g.comm_create(3, 2)
     with pytest.raises(la.LocalAdaAlterError):
         g.set_worker_range(7, 8)
+
+
+TWO_PROCESS = r'''
+import os, sys
+sys.path.insert(0, os.environ["LA_ROOT"])
+import numpy as np, torch, torch.distributed as dist
+from paper_1911_09030_b200 import local_adaalter as la
+from paper_1911_09030_b200.worker_sharded import CudaEngine, WorkerShardedJob
+from oracle.oracle import Oracle
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+torch.cuda.set_device(0)                      # both ranks share the one GPU; no kernel waits for the other rank
+n, W_local, H, T = 40000, 4, 3, 8
+rng = np.random.default_rng(0)
+a = rng.uniform(0.1, 10, n).astype(np.float32); c = rng.standard_normal(n).astype(np.float32)
+g = la.LocalAdaAlter([n], W_local, 0.1, 1.0, la.LA_H_NEVER)
+g.set_grad_quadratic(9, a, c, 0.3)
+eng = CudaEngine(g, rank, world)
+eng.attach_peers(dist)                        # CUDA IPC handles through the process group
+job = WorkerShardedJob(eng, H, exchange="peer", dist=dist)
+job.run(T)
+g.stream_sync()
+mine = [g.read_state(i) for i in range(W_local)]
+parts = [None] * world
+dist.all_gather_object(parts, (rank, mine, g.get_counters()))
+dist.barrier()
+if rank == 0:
+    o = Oracle(n, W_local * world, 0.1, 1.0, H)
+    o.set_grad_quadratic(9, a, c, 0.3)
+    o.run(T)
+    for r, st, cnt in parts:
+        assert cnt == o.counters()
+        for i in range(W_local):
+            for u, v in zip(st[i], o.read(r * W_local + i)):
+                assert np.array_equal(u.view(np.uint32), v.view(np.uint32)), (r, i)
+    print("IPC_PEER_OK")
+g.close()
+dist.destroy_process_group()
+'''
+
+
+def test_two_processes_exchange_through_cuda_ipc(tmp_path):
+    """Two OS processes (gloo for the host-side barriers and the handle exchange) map each other's
+    exchange buffer with CUDA IPC and synchronise with the peer-load combine kernel; the result is
+    the oracle's with W_total workers, bitwise.  Both processes use the same GPU here."""
+    import os, socket, subprocess, sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    script = tmp_path / "ipc_worker.py"
+    script.write_text(TWO_PROCESS)
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    env = dict(os.environ, LA_ROOT=root, MASTER_ADDR="127.0.0.1")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), str(script)]
+    r = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-4000:]
+    assert "IPC_PEER_OK" in r.stdout
