@@ -11,9 +11,14 @@
 #pragma once
 #include "la_sweep.cuh"
 
+#ifndef LA_PERIOD_UNROLL
+#define LA_PERIOD_UNROLL 2
+#endif
+
 namespace la {
 
-constexpr int kPeriodMax = 8;  // steps per pass; step sizes r_s of a group stay in registers
+constexpr int kPeriodMax = 8;  // steps per pass
+constexpr int kPeriodUnroll = LA_PERIOD_UNROLL;
 
 struct PeriodParams {
   SweepParams base;  // base.t = global step BEFORE the first of the h steps, base.tp = t' before it
@@ -32,6 +37,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_period(const PeriodParams p
   // stream keys of every (step, worker) of this pass, and the per-step scalars
   __shared__ uint64_t keys[kPeriodMax][kMaxWorkers];
   __shared__ float eta_s[kPeriodMax], q_s[kPeriodMax];
+  __shared__ Vec<V> r_s[kPeriodMax][LA_BLOCK];
   if (kNeedsNoise) {
     for (uint32_t k = threadIdx.x; k < h * W; k += blockDim.x) {
       const uint32_t s = k / W, i = k - s * W;
@@ -73,11 +79,11 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_period(const PeriodParams p
     const uint64_t ctr0 = kGoldenGamma * (((p.j_base + off) >> 1) + 1u);
     uint64_t st_addr = x_base + off * sizeof(float);
 
-    // step sizes of the h steps: the stale accumulator is fixed, only t' eps^2 ramps
-    Vec<V> r[kPeriodMax];
-#pragma unroll
-    for (int s = 0; s < kPeriodMax; ++s)
-      if (s < (int)h) r[s] = step_size<V>(in.bs, q_s[s], eta_s[s]);
+    // step sizes of the h steps: the stale accumulator is fixed, only t' eps^2 ramps.  They live
+    // in this thread's own shared-memory column so that the loop over steps can stay rolled: with
+    // it unrolled the kernel body (W x 8 copies of the gradient source) overflowed the
+    // instruction cache and a fifth of the issue slots went to instruction-fetch stalls.
+    for (uint32_t s = 0; s < h; ++s) r_s[s][threadIdx.x] = step_size<V>(in.bs, q_s[s], eta_s[s]);
     PairTree<V> tree;
 
 #pragma unroll kOuterUnroll
@@ -95,12 +101,11 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_period(const PeriodParams p
       for (int k = 0; k < CH; ++k)
         if (i0 + k < W) {
           const uint32_t i = i0 + k;
-#pragma unroll
-          for (int s = 0; s < kPeriodMax; ++s)
-            if (s < (int)h) {
-              const Vec<V> g = gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[s][i] : 0ull, ctr0, i, off);
-              apply<V>(r[s], g, cur.x[k], cur.b[k]);
-            }
+#pragma unroll kPeriodUnroll
+          for (uint32_t s = 0; s < h; ++s) {
+            const Vec<V> g = gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[s][i] : 0ull, ctr0, i, off);
+            apply<V>(r_s[s][threadIdx.x], g, cur.x[k], cur.b[k]);
+          }
           if (POST) {
             tree.push(i, cur.x[k], cur.b[k]);
           } else {
