@@ -376,3 +376,35 @@ def test_profiling_stats():
     assert st["ms_local"] > 0 and st["ms_sync"] > 0
     assert st["bytes_local"] == 8 * (16 * 4 + 4) * (1 << 16)
     assert st["bytes_sync"] == 2 * (16 * 4 + 4) * (1 << 16)
+
+
+@pytest.mark.parametrize("W,n", [(4, 1000), (16, 65), (3, 4097), (8, 1)])
+def test_no_write_outside_the_arena(W, n):
+    """Guard bands around a caller-provided arena stay untouched by every kernel of the path
+    (the stand-in for a memory checker: the kernels index only inside la_arena_bytes)."""
+    import torch
+    need = la.LocalAdaAlter.arena_bytes([n], W) // 4
+    guard = 4096                                                   # floats on each side (256-byte multiple)
+    buf = torch.full((need + 2 * guard,), -777.0, dtype=torch.float32, device="cuda")
+    assert buf.data_ptr() % 256 == 0
+    arena = buf[guard:guard + need]
+    arr = _arrays(n, 9)
+    g = la.LocalAdaAlter([n], W, 0.1, 1.0, 3, arena=arena, device=torch.cuda.current_device())
+    g.set_grad_quadratic(4, arr["a"], arr["c"], 0.5)
+    for fusion in (0, 1, 2, 3):
+        g.set_fusion(fusion)
+        g.run(7)
+    g.set_grad_noise(4, arr["s"]); g.run(4)
+    g.set_grad_dtype(la.LA_BF16); g.run(3); g.set_grad_dtype(la.LA_F32)
+    G = torch.randn(W * n, device="cuda")
+    g.step_grads(G.data_ptr(), la.LA_F32)
+    g.step_grads(G.to(torch.bfloat16).data_ptr(), la.LA_BF16)
+    g.sync()
+    g.set_rule(la.LA_RULE_LOCAL_SGD); g.run(6)
+    g.set_rule(la.LA_RULE_ADAGRAD); g.run(3)
+    g.set_rule(la.LA_RULE_ADAALTER)
+    g.set_init(None, 0.5)
+    g.sync_stream()
+    torch.cuda.synchronize()
+    assert bool((buf[:guard] == -777.0).all()) and bool((buf[guard + need:] == -777.0).all())
+    g.close()
