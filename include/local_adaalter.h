@@ -207,6 +207,22 @@ int la_comm_set_peer(la_ctx* ctx, uint32_t peer_rank, void* dev_ptr);
 int la_comm_export(la_ctx* ctx);
 int la_comm_combine(la_ctx* ctx);
 int la_comm_import(la_ctx* ctx);
+/* The local steps next to a synchronisation, fused with the exchange, so that the
+ * synchronisation costs no pass over the replicas of its own:
+ *   la_comm_step_export        the local step of Algorithm 3 (generated gradients) that completes a
+ *                              period; its y and A^2 are not stored (the means will replace them),
+ *                              only their tree sums go to the exchange buffer.  t += 1, t' += 1.
+ *                              Until the import the replicas hold the PREVIOUS step's values.
+ *   la_comm_step_grads_export  the same with caller-supplied gradients (table as for
+ *                              la_local_step_grads)
+ *   la_comm_import_step        la_comm_import and the first local step of the next period in one
+ *                              pass: every replica starts from total / W_total.  n_sync += 1,
+ *                              t += 1, t' = 1.  (With H = 1 use la_comm_import instead.)
+ * Sequence: step_export, exchange (la_comm_combine between barriers, or an all-reduce of the
+ * buffer), then import_step or import.  Results are bitwise those of the unfused calls. */
+int la_comm_step_export(la_ctx* ctx);
+int la_comm_step_grads_export(la_ctx* ctx, const void* g_dev, int dtype);
+int la_comm_import_step(la_ctx* ctx);
 /* Block until the context's stream is idle. */
 int la_stream_sync(la_ctx* ctx);
 

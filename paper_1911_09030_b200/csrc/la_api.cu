@@ -54,6 +54,33 @@ PeriodKernel lookup_period(int W, int gm, bool bf16, bool post) {
   }
 }
 
+#define LA_DECL_XCH(w)                                   \
+  StepExportFn lookup_step_export_w##w(int, bool);       \
+  ImportStepFn lookup_import_step_w##w(int, bool);
+LA_DECL_XCH(0) LA_DECL_XCH(1) LA_DECL_XCH(2) LA_DECL_XCH(4) LA_DECL_XCH(8) LA_DECL_XCH(16)
+#undef LA_DECL_XCH
+
+StepExportFn lookup_step_export(int W, int gm, bool bf16) {
+  switch (W) {
+    case 1: return lookup_step_export_w1(gm, bf16);
+    case 2: return lookup_step_export_w2(gm, bf16);
+    case 4: return lookup_step_export_w4(gm, bf16);
+    case 8: return lookup_step_export_w8(gm, bf16);
+    case 16: return lookup_step_export_w16(gm, bf16);
+    default: return lookup_step_export_w0(gm, bf16);
+  }
+}
+ImportStepFn lookup_import_step(int W, int gm, bool bf16) {
+  switch (W) {
+    case 1: return lookup_import_step_w1(gm, bf16);
+    case 2: return lookup_import_step_w2(gm, bf16);
+    case 4: return lookup_import_step_w4(gm, bf16);
+    case 8: return lookup_import_step_w8(gm, bf16);
+    case 16: return lookup_import_step_w16(gm, bf16);
+    default: return lookup_import_step_w0(gm, bf16);
+  }
+}
+
 ExchangeFn lookup_export_w0();
 ExchangeFn lookup_export_w1();
 ExchangeFn lookup_export_w2();
@@ -887,6 +914,78 @@ int la_comm_import(la_ctx* c) {
   LA_CUDA(c, cudaGetLastError());
   c->stats.launches_other++;
   c->tp = 0; c->nsync += 1;
+  return LA_OK;
+}
+
+// Parameters of a step launched outside launch_sweep (the exchange-fused steps).
+static void step_params(const la_ctx* c, la::SweepParams* p, uint64_t t, uint32_t tp, const void* gext, int gm) {
+  std::memset(p, 0, sizeof *p);
+  p->X = c->X; p->B2 = c->B2; p->Bs = c->Bs;
+  p->a = c->pa; p->c = c->pc; p->s = c->has_s ? c->ps : nullptr;
+  p->gext = gext;
+  if (gext) {
+    const uint64_t elem = (gm == la::kGradExternalBF16) ? 2 : 4;
+    p->gext_vec = (c->N % kExchangeVecHost == 0 && (reinterpret_cast<uintptr_t>(gext) % (kExchangeVecHost * elem)) == 0) ? 1u : 0u;
+  }
+  p->n = c->N; p->stride = c->stride; p->j_base = c->j_base;
+  p->seed = c->seed; p->t = t; p->W = c->W; p->tp = tp;
+  p->warm_up_steps = c->warm_up_steps; p->identical_workers = c->identical ? 1u : 0u;
+  p->worker_base = c->worker_base;
+  p->eta = c->eta; p->eps = c->eps; p->sigma = c->sigma;
+}
+
+static unsigned step_grid(const la_ctx* c) {
+  const uint64_t groups = (c->N + kExchangeVecHost - 1) / kExchangeVecHost;
+  uint64_t blocks = (groups + la::kBlockThreads - 1) / la::kBlockThreads;
+  const uint64_t cap = (uint64_t)c->num_sms * (uint64_t)(c->blocks_per_sm > 0 ? c->blocks_per_sm : 96);
+  if (blocks > cap) blocks = cap;
+  return blocks ? (unsigned)blocks : 1u;
+}
+
+static int step_export_impl(la_ctx* c, int gm, const void* gext) {
+  if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
+  if (c->rule != LA_RULE_ADAALTER) return fail(c, LA_ESTATE, "sharding by worker is implemented for Local AdaAlter only");
+  const bool bf16 = c->bf16 && gm <= la::kGradQuadratic;
+  la::StepExportFn fn = la::lookup_step_export((int)c->W, gm, bf16);
+  if (!fn) return fail(c, LA_ESTATE, "no step+export kernel for this combination (W=%u grad=%d)", c->W, gm);
+  DeviceGuard guard(c->device);
+  la::SweepParams p;
+  step_params(c, &p, c->t + 1, c->tp + 1, gext, gm);
+  fn<<<step_grid(c), la::kBlockThreads, 0, c->stream>>>(p, c->S);
+  LA_CUDA(c, cudaGetLastError());
+  c->stats.launches_fused++;
+  c->stats.bytes_fused += 8.0 * c->W * (double)c->N + pass_bytes(c, false, true, false, gm) - 16.0 * c->W * (double)c->N + 8.0 * (double)c->N;
+  c->t += 1; c->tp += 1;
+  return LA_OK;
+}
+
+int la_comm_step_export(la_ctx* c) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  return step_export_impl(c, c->grad_kind, nullptr);
+}
+
+int la_comm_step_grads_export(la_ctx* c, const void* g_dev, int dtype) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!g_dev) return fail(c, LA_EINVAL, "g_dev is NULL");
+  if (dtype != LA_F32 && dtype != LA_BF16) return fail(c, LA_EINVAL, "dtype must be LA_F32 or LA_BF16");
+  return step_export_impl(c, dtype == LA_F32 ? la::kGradExternalF32 : la::kGradExternalBF16, g_dev);
+}
+
+int la_comm_import_step(la_ctx* c) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
+  if (c->rule != LA_RULE_ADAALTER) return fail(c, LA_ESTATE, "sharding by worker is implemented for Local AdaAlter only");
+  const bool bf16 = c->bf16 && c->grad_kind <= la::kGradQuadratic;
+  la::ImportStepFn fn = la::lookup_import_step((int)c->W, c->grad_kind, bf16);
+  if (!fn) return fail(c, LA_ESTATE, "no import+step kernel for this combination (W=%u grad=%d)", c->W, c->grad_kind);
+  DeviceGuard guard(c->device);
+  la::SweepParams p;
+  step_params(c, &p, c->t + 1, 1u, nullptr, c->grad_kind);
+  fn<<<step_grid(c), la::kBlockThreads, 0, c->stream>>>(p, c->S, c->W_total);
+  LA_CUDA(c, cudaGetLastError());
+  c->stats.launches_fused++;
+  c->stats.bytes_fused += pass_bytes(c, true, true, false, c->grad_kind) - 8.0 * c->W * (double)c->N + 8.0 * (double)c->N;
+  c->nsync += 1; c->t += 1; c->tp = 1;
   return LA_OK;
 }
 

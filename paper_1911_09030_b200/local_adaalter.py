@@ -88,6 +88,9 @@ def lib() -> C.CDLL:
             "la_comm_export": [vp],
             "la_comm_combine": [vp],
             "la_comm_import": [vp],
+            "la_comm_step_export": [vp],
+            "la_comm_step_grads_export": [vp, vp, i32],
+            "la_comm_import_step": [vp],
             "la_stream_sync": [vp],
             "la_replica_means_static": [vp, vp, u32, u64, u64, vp, vp, vp],
         }
@@ -346,3 +349,12 @@ class LocalAdaAlter:
 
     def comm_import(self):
         self._ck(self.L.la_comm_import(self.h))
+
+    def comm_step_export(self):
+        self._ck(self.L.la_comm_step_export(self.h))
+
+    def comm_step_grads_export(self, g_dev_ptr, dtype=LA_F32):
+        self._ck(self.L.la_comm_step_grads_export(self.h, C.c_void_p(int(g_dev_ptr)), int(dtype)))
+
+    def comm_import_step(self):
+        self._ck(self.L.la_comm_import_step(self.h))

@@ -20,10 +20,14 @@ from typing import Optional
 
 
 class WorkerShardedJob:
-    def __init__(self, engine, H: int, exchange: str = "peer", dist=None, group=None):
+    def __init__(self, engine, H: int, exchange: str = "peer", dist=None, group=None, fused: bool = False):
+        """fused=True: the step that completes a period writes only its sums to the exchange buffer
+        and the first step of the next period starts from the exchanged totals, so a
+        synchronisation adds no pass over the replicas (engine needs step_export/import_step)."""
         if exchange not in ("peer", "allreduce"):
             raise ValueError("exchange must be 'peer' or 'allreduce'")
         self.engine, self.H, self.exchange, self.dist, self.group = engine, int(H), exchange, dist, group
+        self.fused = bool(fused) and self.H > 1
         self.syncs = 0
 
     def _barrier(self):
@@ -31,8 +35,13 @@ class WorkerShardedJob:
             self.dist.barrier(group=self.group)
 
     def sync(self):
+        self.engine.export()
+        self._exchange()
+        self.engine.import_()
+        self.syncs += 1
+
+    def _exchange(self):
         e = self.engine
-        e.export()
         if self.exchange == "peer":
             e.stream_sync()
             self._barrier()            # every rank's sums are in its buffer
@@ -43,15 +52,26 @@ class WorkerShardedJob:
             buf = e.buffer_tensor()
             if self.dist is not None and self.dist.is_initialized() and self.dist.get_world_size(self.group) > 1:
                 self.dist.all_reduce(buf, op=self.dist.ReduceOp.SUM, group=self.group)
-        e.import_()
-        self.syncs += 1
 
     def run(self, T: int):
         """T iterations of Algorithm 3: local step; if t' == H: synchronise."""
-        for _ in range(int(T)):
-            self.engine.local_step()
-            if self.engine.t_prime() == self.H:
-                self.sync()
+        e, k, T = self.engine, 0, int(T)
+        while k < T:
+            if self.fused and e.t_prime() + 1 == self.H:
+                e.step_export()                 # iteration k: the step that completes the period
+                self._exchange()
+                k += 1
+                if k < T:
+                    e.import_step()             # iteration k+1 starts from the exchanged means
+                    k += 1
+                else:
+                    e.import_()
+                self.syncs += 1
+            else:
+                e.local_step()
+                k += 1
+                if e.t_prime() == self.H:
+                    self.sync()
 
 
 class _DeviceBuffer:
@@ -93,6 +113,12 @@ class CudaEngine:
 
     def import_(self):
         self.ctx.comm_import()
+
+    def step_export(self):
+        self.ctx.comm_step_export()
+
+    def import_step(self):
+        self.ctx.comm_import_step()
 
     def stream_sync(self):
         self.ctx.stream_sync()

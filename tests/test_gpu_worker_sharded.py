@@ -169,3 +169,102 @@ def test_two_processes_exchange_through_cuda_ipc(tmp_path):
     r = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=300)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-4000:]
     assert "IPC_PEER_OK" in r.stdout
+
+
+@pytest.mark.parametrize("H,T", [(2, 9), (3, 10), (4, 8), (5, 5), (1, 4)])
+def test_fused_exchange_steps_with_one_rank(H, T):
+    n, W = 30001, 8
+    a, c = _arrays(n, H)
+    ref = _single(n, W, H, a, c, T)
+    g = la.LocalAdaAlter([n], W, 0.1, 1.0, la.LA_H_NEVER)
+    g.set_grad_quadratic(9, a, c, 0.3)
+    job = WorkerShardedJob(CudaEngine(g, 0, 1), H, exchange="peer", fused=True)
+    job.run(3)
+    job.run(T - 3)
+    assert g.get_counters() == ref.get_counters()
+    assert job.syncs == T // H
+    for i in range(W):
+        for u, v in zip(g.read_state(i), ref.read_state(i)):
+            assert np.array_equal(u.view(np.uint32), v.view(np.uint32))
+    if H > 1:
+        st = g.get_stats()
+        assert st["launches_fused"] >= T // H          # step+export / import+step kernels were used
+
+
+@pytest.mark.parametrize("world,W_local,grad", [(2, 4, "quadratic"), (4, 2, "noise"), (2, 8, "supplied")])
+def test_fused_exchange_steps_with_emulated_ranks(world, W_local, grad):
+    import torch
+    n, H, T = 6002, 3, 8
+    W_total = world * W_local
+    a, c = _arrays(n, 5)
+    o = Oracle(n, W_total, 0.1, 1.0, H)
+    ctxs = []
+    for r in range(world):
+        g = la.LocalAdaAlter([n], W_local, 0.1, 1.0, la.LA_H_NEVER)
+        g.comm_create(r, world)
+        ctxs.append(g)
+    if grad == "quadratic":
+        o.set_grad_quadratic(9, a, c, 0.3)
+        for g in ctxs:
+            g.set_grad_quadratic(9, a, c, 0.3)
+    elif grad == "noise":
+        o.set_grad_noise(9, None)
+        for g in ctxs:
+            g.set_grad_noise(9, None)
+    for r in range(world):
+        for q in range(world):
+            if q != r:
+                ctxs[r].comm_set_peer(q, ctxs[q].comm_buffer()[0])
+    rng = np.random.default_rng(1)
+
+    def exchange():
+        for g in ctxs:
+            g.stream_sync()
+        for g in ctxs:
+            g.comm_combine()
+        for g in ctxs:
+            g.stream_sync()
+
+    t = 0
+    while t < T:
+        closes = (ctxs[0].get_counters()[1] + 1 == H)
+        if grad == "supplied":
+            G = rng.standard_normal((W_total, n)).astype(np.float32)
+            o.local_step(G)
+            for r, g in enumerate(ctxs):
+                Gd = torch.from_numpy(G[r * W_local:(r + 1) * W_local].copy()).cuda()
+                if closes:
+                    g.comm_step_grads_export(Gd.data_ptr(), la.LA_F32)
+                else:
+                    g.local_step_grads(Gd.data_ptr(), la.LA_F32)
+                g.stream_sync()
+            t += 1
+            if closes:
+                exchange()
+                for g in ctxs:
+                    g.comm_import()
+                o.sync()
+            continue
+        if closes:
+            for g in ctxs:
+                g.comm_step_export()
+            exchange()
+            t += 1
+            if t < T:
+                for g in ctxs:
+                    g.comm_import_step()
+                t += 1
+            else:
+                for g in ctxs:
+                    g.comm_import()
+        else:
+            for g in ctxs:
+                g.local_step()
+            t += 1
+    if grad != "supplied":
+        o.run(T)
+    for r, g in enumerate(ctxs):
+        assert g.get_counters() == o.counters()
+        for i in range(W_local):
+            for name, u, w in zip("x b2 bs".split(), g.read_state(i), o.read(r * W_local + i)):
+                assert np.array_equal(u.view(np.uint32), w.view(np.uint32)), f"{name} rank {r} worker {i}"
