@@ -359,8 +359,9 @@ int launch_period(la_ctx* c, uint32_t h, bool post) {
   const unsigned block = la::kBlockThreads;
   const uint64_t ngroups = (c->N + (uint64_t)k.vec - 1) / (uint64_t)k.vec;
   uint64_t blocks = (ngroups + block - 1) / block;
-  // issue-bound kernel: measured optimum around 192 blocks per SM in the grid (sweep 12..4096)
-  const int bps = c->blocks_per_sm > 0 ? c->blocks_per_sm : 192;
+  // issue-bound kernel: at the full configuration sizes 384..768 blocks per SM in the grid measured
+  // best (few coordinate groups per thread); smaller grids lose up to 20 %
+  const int bps = c->blocks_per_sm > 0 ? c->blocks_per_sm : 768;
   const uint64_t cap = (uint64_t)c->num_sms * (uint64_t)bps;
   if (blocks > cap) blocks = cap;
   EventPair ep{};
@@ -680,7 +681,9 @@ int la_run(la_ctx* c, uint64_t T) {
       if (h > left) h = left;
       if (h > (uint64_t)la::kPeriodMax) h = la::kPeriodMax;
       const bool closes = (c->tp + h == c->H);
-      int rc = launch_period(c, (uint32_t)h, closes);
+      // a single step gains nothing from the blocked kernel: use the step kernels (K1 / K3)
+      int rc = (h == 1) ? launch_sweep(c, false, true, closes, c->t + 1, c->tp + 1, c->grad_kind, nullptr)
+                        : launch_period(c, (uint32_t)h, closes);
       if (rc) return rc;
       c->t += h;
       if (closes) { c->tp = 0; c->nsync += 1; } else { c->tp += (uint32_t)h; }

@@ -105,8 +105,10 @@ def test_fused_kernels_equal_unfused_bitwise(W, H):
     assert states[1][2]["launches_fused"] == T // H and states[1][2]["launches_sync"] == 0
     assert states[2][2]["launches_fused"] > 0
     # temporal blocking: one pass per (piece of a) period, nothing else
-    assert states[3][2]["launches_local"] == 0 and states[3][2]["launches_sync"] == 0
-    assert states[3][2]["launches_fused"] <= -(-4 // min(H, 8)) + -(-(T - 4) // min(H, 8)) + 2
+    # (a piece of a single step runs as an ordinary step kernel), never a stand-alone sync
+    assert states[3][2]["launches_sync"] == 0
+    assert states[3][2]["launches_fused"] + states[3][2]["launches_local"] <= \
+        -(-4 // min(H, 8)) + -(-(T - 4) // min(H, 8)) + 2
 
 
 # ----------------------------------------------------------------------------- schedule
