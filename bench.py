@@ -208,12 +208,13 @@ def run_ours(args, wl):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local_rank)
-    if world > 1:
+    use_dist = world > 1 or ("RANK" in os.environ and "MASTER_PORT" in os.environ)   # launched by torchrun
+    if use_dist:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     def barrier():
-        if world > 1:
+        if use_dist:
             dist.barrier()
         torch.cuda.synchronize()
 
@@ -287,7 +288,7 @@ def run_ours(args, wl):
         p1.record(stream)
         barrier()
         pst = ctx.get_stats(reset=True)
-        pms = sharding.max_over_ranks(p0.elapsed_time(p1) / args.steps, dist if world > 1 else None)
+        pms = sharding.max_over_ranks(p0.elapsed_time(p1) / args.steps, dist if use_dist else None)
         period = {"ms_per_step": pms, "value": wl.W * wl.N * wl.T * world / (pms * 1e-3), "unit": UNIT,
                   "launches_per_step": pst["launches_fused"] // args.steps,
                   "hbm_GBps": pst["bytes_fused"] / args.steps / (pms * 1e-3) / 1e9}
@@ -308,8 +309,8 @@ def run_ours(args, wl):
     barrier()
     e2e_ms = 1e3 * (time.perf_counter() - t0) / e2e_steps
 
-    ms_total = sharding.max_over_ranks(ms_total, dist if world > 1 else None)
-    e2e_ms = sharding.max_over_ranks(e2e_ms, dist if world > 1 else None)
+    ms_total = sharding.max_over_ranks(ms_total, dist if use_dist else None)
+    e2e_ms = sharding.max_over_ranks(e2e_ms, dist if use_dist else None)
     ms_per_step = ms_total / args.steps
     units = wl.W * wl.N * wl.T * world
     value = units / (ms_per_step * 1e-3)
@@ -365,7 +366,7 @@ def run_ours(args, wl):
         }
         print(json.dumps(line), flush=True)
     ctx.close()
-    if world > 1:
+    if use_dist:
         dist.destroy_process_group()
 
 

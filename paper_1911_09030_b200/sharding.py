@@ -36,7 +36,7 @@ def weak_scaling_base(N: int, rank: int, align: int = ALIGN) -> int:
 
 def max_over_ranks(value: float, dist=None) -> float:
     """Max of a per-rank scalar (e.g. a device-timed duration); identity without a process group."""
-    if dist is None or not dist.is_available() or not dist.is_initialized() or dist.get_world_size() == 1:
+    if dist is None or not dist.is_available() or not dist.is_initialized():
         return float(value)
     import torch
     dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
