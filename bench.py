@@ -458,6 +458,56 @@ def run_report(args):
               f"{f2(r['us_fused'], 1)} ({f2(r['GBps_fused'])}) | {f2(100 * r['sync_share_of_time'], 1)} % |")
 
 
+def run_tradeoff(args):
+    """Single-GPU analogue of the paper's Table 2 (quality and time against the synchronisation
+    period): the noisy quadratic of configuration 3 at N = 2^24, T = 256 iterations, for Local
+    AdaAlter with H in {1,4,8,16,64,never} (unfused, so that the synchronisation cost is visible,
+    and fused) and for the two baseline rules.  Prints objective at the mean iterate, replica
+    spread before the last synchronisation, and time."""
+    import torch
+    from paper_1911_09030_b200 import local_adaalter as la
+    from paper_1911_09030_b200 import workloads
+    torch.cuda.set_device(0)
+    wl = workloads.config("c3")
+    wl.sizes = [1 << 24]
+    arr = wl.arrays()
+    T = 256
+    rows = []
+
+    def one(label, rule, H, fusion):
+        ctx = la.LocalAdaAlter.with_torch_arena(wl.sizes, wl.W, wl.eta, wl.eps, H, b0sq=1.0)
+        ctx.set_init(None, 1.0)
+        ctx.set_grad_quadratic(wl.noise_seed, arr["a"], arr["c"], wl.sigma)
+        ctx.set_rule(rule)
+        ctx.set_fusion(fusion)
+        f0 = ctx.diagnostics()[0]
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        st = torch.cuda.current_stream()
+        e0.record(st)
+        ctx.run(T - 1)
+        e1.record(st)
+        torch.cuda.synchronize()
+        spread = ctx.diagnostics()[1]
+        ctx.run(1)
+        f = ctx.diagnostics()[0]
+        rows.append((label, H, fusion, f / f0, spread / wl.N, e0.elapsed_time(e1) * T / (T - 1), ctx.get_counters()[2]))
+        ctx.close()
+
+    for H in (1, 4, 8, 16, 64, la.LA_H_NEVER):
+        one("Local AdaAlter", la.LA_RULE_ADAALTER, H, 0)
+    for H in (4, 16):
+        one("Local AdaAlter", la.LA_RULE_ADAALTER, H, 1)
+        one("Local AdaAlter", la.LA_RULE_ADAALTER, H, 3)
+    one("Distributed AdaGrad", la.LA_RULE_ADAGRAD, 1, 0)
+    for H in (1, 16):
+        one("Local SGD", la.LA_RULE_LOCAL_SGD, H, 0)
+    print("| rule | H | fusion | F(x-bar_T)/F(x_0) | replica spread per coordinate at T-1 | ms for T=256 | exchanges |")
+    print("|---|---|---|---|---|---|---|")
+    for label, H, fusion, f, sp, ms, ns in rows:
+        hs = "never" if H == la.LA_H_NEVER else str(H)
+        print(f"| {label} | {hs} | {fusion} | {f:.5f} | {sp:.3e} | {ms:.1f} | {ns} |")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -474,11 +524,14 @@ def main():
     ap.add_argument("--no-period", action="store_true", help="skip the extra temporal-blocking measurement")
     ap.add_argument("--report", action="store_true", help="all configurations + the H sweep (not the JSON line)")
     ap.add_argument("--report-out", default=None)
+    ap.add_argument("--tradeoff", action="store_true", help="quality/time against H on a noisy quadratic (table)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     if args.report:
         return run_report(args)
+    if args.tradeoff:
+        return run_tradeoff(args)
     from paper_1911_09030_b200 import workloads
     wl = workloads.config(args.workload)
     if args.H is not None:

@@ -175,6 +175,15 @@ int la_set_counters(la_ctx* ctx, uint64_t t, uint32_t t_prime, uint64_t n_sync);
  * reset != 0 clears the counters after reading. */
 int la_get_stats(la_ctx* ctx, la_stats* out, int reset);
 
+/* Diagnostics, off the hot path (synchronises the stream; its first call allocates 16 bytes of
+ * device memory).  With x-bar the mean iterate over workers (the auxiliary sequence of Section 5):
+ *   objective      = 1/2 sum_j a_j (x-bar_j - c_j)^2, the noisy-quadratic objective at x-bar
+ *                    (NaN unless the quadratic gradient source is set)
+ *   replica_spread = (1/W) sum_i ||x_i - x-bar||^2, the drift of the replicas since the last
+ *                    synchronisation (the quantity Appendix A bounds through H); 0 right after a sync
+ * Accumulated in double.  Either pointer may be NULL. */
+int la_diagnostics(la_ctx* ctx, double* objective, double* replica_spread);
+
 /* ---- sharding BY WORKER across GPUs (one process per GPU) -----------------------------------
  * The layout of the paper: the workers of Algorithm 3 sit on different devices and exchange x
  * and B^2 every H steps (Section 4.2).  A rank holds W (local) replicas out of W_total.

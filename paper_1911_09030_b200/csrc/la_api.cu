@@ -113,6 +113,53 @@ __global__ void la_fill(float* X, float* B2, float* Bs, const float* x0, float b
   }
 }
 
+// Diagnostics (off the hot path): with x-bar = mean over workers (plain left-to-right sum in
+// double), out[0] += sum_j a_j (x-bar_j - c_j)^2 / 2  (the quadratic objective at the mean iterate,
+// the quantity whose gradient norm Theorem 1 bounds) and out[1] += sum_i sum_j (x_ij - x-bar_j)^2 / W
+// (how far the replicas have drifted apart since the last synchronisation; the term the proof
+// in Appendix A controls by H).  a == nullptr skips the objective.
+__global__ void la_diagnostics(const float* __restrict__ X, const float* __restrict__ a, const float* __restrict__ c,
+                               uint64_t n, uint64_t stride, uint32_t W, double* __restrict__ out) {
+  double f = 0.0, d = 0.0;
+  const uint64_t nthreads = (uint64_t)gridDim.x * blockDim.x;
+  for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += nthreads) {
+    double m = 0.0;
+    for (uint32_t i = 0; i < W; ++i) m += (double)X[(uint64_t)i * stride + j];
+    m /= (double)W;
+    double dev = 0.0;
+    for (uint32_t i = 0; i < W; ++i) {
+      const double e = (double)X[(uint64_t)i * stride + j] - m;
+      dev += e * e;
+    }
+    d += dev / (double)W;
+    if (a != nullptr) {
+      const double e = m - (double)c[j];
+      f += 0.5 * (double)a[j] * e * e;
+    }
+  }
+  // block reduction, then one atomic pair per block
+  __shared__ double sf[LA_BLOCK / 32], sd[LA_BLOCK / 32];
+  for (int o = 16; o > 0; o >>= 1) {
+    f += __shfl_down_sync(0xffffffffu, f, o);
+    d += __shfl_down_sync(0xffffffffu, d, o);
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) { sf[warp] = f; sd[warp] = d; }
+  __syncthreads();
+  if (warp == 0) {
+    f = lane < (int)(blockDim.x >> 5) ? sf[lane] : 0.0;
+    d = lane < (int)(blockDim.x >> 5) ? sd[lane] : 0.0;
+    for (int o = 16; o > 0; o >>= 1) {
+      f += __shfl_down_sync(0xffffffffu, f, o);
+      d += __shfl_down_sync(0xffffffffu, d, o);
+    }
+    if (lane == 0) {
+      atomicAdd(out, f);
+      atomicAdd(out + 1, d);
+    }
+  }
+}
+
 }  // namespace la
 
 namespace {
@@ -156,6 +203,7 @@ struct la_ctx {
   float* S = nullptr;
   float* peerS[la::kMaxRanks] = {};
   void* ipc_opened[la::kMaxRanks] = {};
+  double* diag = nullptr;  // two doubles for la_diagnostics, allocated on its first call
   // schedule (Algorithm 3): t = local steps so far, tp = local steps since the last sync
   uint64_t t = 0, nsync = 0;
   uint32_t tp = 0;
@@ -497,6 +545,7 @@ void la_destroy(la_ctx* c) {
   for (auto& p : c->pool) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
   for (auto*& m : c->ipc_opened) if (m) { cudaIpcCloseMemHandle(m); m = nullptr; }
   if (c->S) cudaFree(c->S);
+  if (c->diag) cudaFree(c->diag);
   if (c->owns_arena && c->arena) cudaFree(c->arena);
   delete c;
 }
@@ -989,6 +1038,31 @@ int la_comm_import_step(la_ctx* c) {
   c->stats.launches_fused++;
   c->stats.bytes_fused += pass_bytes(c, true, true, false, c->grad_kind) - 8.0 * c->W * (double)c->N + 8.0 * (double)c->N;
   c->nsync += 1; c->t += 1; c->tp = 1;
+  return LA_OK;
+}
+
+int la_diagnostics(la_ctx* c, double* objective, double* replica_spread) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  DeviceGuard guard(c->device);
+  if (!c->diag) {
+    cudaError_t e = cudaMalloc((void**)&c->diag, 2 * sizeof(double));
+    if (e != cudaSuccess) { c->diag = nullptr; cudaGetLastError(); return fail(c, LA_ENOMEM, "cudaMalloc failed: %s", cudaGetErrorString(e)); }
+  }
+  LA_CUDA(c, cudaMemsetAsync(c->diag, 0, 2 * sizeof(double), c->stream));
+  const bool quad = c->grad_kind == la::kGradQuadratic;
+  const uint32_t W = c->rule == LA_RULE_ADAGRAD ? 1u : c->W;  // AdaGrad keeps one shared iterate
+  uint64_t blocks = (c->N + la::kBlockThreads - 1) / la::kBlockThreads;
+  const uint64_t cap = (uint64_t)c->num_sms * 16;
+  if (blocks > cap) blocks = cap;
+  la::la_diagnostics<<<(unsigned)blocks, la::kBlockThreads, 0, c->stream>>>(c->X, quad ? c->pa : nullptr, c->pc, c->N,
+                                                                             c->stride, W, c->diag);
+  LA_CUDA(c, cudaGetLastError());
+  c->stats.launches_other++;
+  double host[2] = {0, 0};
+  LA_CUDA(c, cudaMemcpyAsync(host, c->diag, sizeof host, cudaMemcpyDeviceToHost, c->stream));
+  LA_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (objective) *objective = quad ? host[0] : NAN;
+  if (replica_spread) *replica_spread = host[1];
   return LA_OK;
 }
 

@@ -79,6 +79,7 @@ def lib() -> C.CDLL:
             "la_get_counters": [vp, C.POINTER(u64), C.POINTER(u32), C.POINTER(u64)],
             "la_set_counters": [vp, u64, u32, u64],
             "la_get_stats": [vp, C.POINTER(la_stats), i32],
+            "la_diagnostics": [vp, C.POINTER(C.c_double), C.POINTER(C.c_double)],
             "la_set_worker_range": [vp, u32, u32],
             "la_comm_create": [vp, u32, u32],
             "la_comm_buffer": [vp, C.POINTER(vp), C.POINTER(u64)],
@@ -309,6 +310,12 @@ class LocalAdaAlter:
         st = la_stats()
         self._ck(self.L.la_get_stats(self.h, C.byref(st), int(bool(reset))))
         return {k: getattr(st, k) for k, _ in la_stats._fields_}
+
+    def diagnostics(self):
+        """(objective at the mean iterate, mean squared distance of the replicas from it)."""
+        f, d = C.c_double(), C.c_double()
+        self._ck(self.L.la_diagnostics(self.h, C.byref(f), C.byref(d)))
+        return f.value, d.value
 
     def sync_stream(self):
         """Block until the context's stream is idle."""

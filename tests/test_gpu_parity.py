@@ -410,3 +410,25 @@ def test_no_write_outside_the_arena(W, n):
     torch.cuda.synchronize()
     assert bool((buf[:guard] == -777.0).all()) and bool((buf[guard + need:] == -777.0).all())
     g.close()
+
+
+def test_diagnostics_objective_and_replica_spread():
+    n, W, H = 5003, 8, 4
+    arr = _arrays(n, 31)
+    g = la.LocalAdaAlter([n], W, 0.1, 1.0, H, b0sq=1.0)
+    g.set_init(None, 1.0)
+    g.set_grad_quadratic(3, arr["a"], arr["c"], 0.5)
+    a, c = arr["a"].astype(np.float64), arr["c"].astype(np.float64)
+    f0, d0 = g.diagnostics()
+    assert f0 == pytest.approx(0.5 * np.sum(a * c * c), rel=1e-12) and d0 == 0.0
+    g.run(6)                                        # two steps into the second period
+    X = np.stack([g.read_state(i)[0] for i in range(W)]).astype(np.float64)
+    xbar = X.mean(0)
+    f, d = g.diagnostics()
+    assert f == pytest.approx(0.5 * np.sum(a * (xbar - c) ** 2), rel=1e-11)
+    assert d == pytest.approx(np.sum((X - xbar) ** 2) / W, rel=1e-11) and d > 0
+    assert f < f0
+    g.run(2)                                        # closes the period: replicas coincide again
+    assert g.diagnostics()[1] == 0.0
+    g.set_grad_noise(1, None)
+    assert np.isnan(g.diagnostics()[0])
