@@ -130,6 +130,13 @@ int la_set_fusion(la_ctx* ctx, int mode);
  * blocks_per_sm * (number of SMs) blocks of 256 threads; 0 restores the built-in
  * per-kernel defaults (96 for kernels that take a step, unbounded for the pure sync). */
 int la_set_launch_shape(la_ctx* ctx, int blocks_per_sm);
+/* Launch-bound regime (small N, e.g. a 2 MB state where a step takes a few microseconds): let
+ * la_run replay whole periods of H iterations from a captured CUDA graph instead of launching
+ * every kernel.  The kernels then read the global step from a device-resident counter, so one
+ * graph serves all periods; results are bitwise unchanged.  Needs a context on a non-default
+ * stream (LA_ESTATE otherwise); allocates 8 bytes on first use; ignored while profiling, for the
+ * AdaGrad rule, for LA_FUSE_SYNC_STEP, and for runs that start inside a period. */
+int la_set_graph(la_ctx* ctx, int on);
 /* Record CUDA events around every launch and accumulate device time per class. */
 int la_set_profiling(la_ctx* ctx, int on);
 

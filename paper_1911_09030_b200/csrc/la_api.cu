@@ -113,6 +113,10 @@ __global__ void la_fill(float* X, float* B2, float* Bs, const float* x0, float b
   }
 }
 
+// Device-resident step counter used by captured graphs (see la_set_graph).
+__global__ void la_counter_set(uint64_t* ctr, uint64_t v) { *ctr = v; }
+__global__ void la_counter_add(uint64_t* ctr, uint64_t v) { *ctr += v; }
+
 // Diagnostics (off the hot path): with x-bar = mean over workers (plain left-to-right sum in
 // double), out[0] += sum_j a_j (x-bar_j - c_j)^2 / 2  (the quadratic objective at the mean iterate,
 // the quantity whose gradient norm Theorem 1 bounds) and out[1] += sum_i sum_j (x_ij - x-bar_j)^2 / W
@@ -204,6 +208,13 @@ struct la_ctx {
   float* peerS[la::kMaxRanks] = {};
   void* ipc_opened[la::kMaxRanks] = {};
   double* diag = nullptr;  // two doubles for la_diagnostics, allocated on its first call
+  // CUDA-graph replay of whole periods (la_set_graph)
+  bool use_graph = false, capturing = false;
+  uint64_t* sched = nullptr;       // device: global step count before the period being replayed
+  uint64_t capture_base = 0;
+  cudaGraphExec_t graph_exec = nullptr;
+  uint64_t graph_key[8] = {};
+  la_stats graph_delta{};          // what one replay adds to the statistics
   // schedule (Algorithm 3): t = local steps so far, tp = local steps since the last sync
   uint64_t t = 0, nsync = 0;
   uint32_t tp = 0;
@@ -356,7 +367,9 @@ int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t
     p.gext_vec = (c->N % (uint64_t)k.vec == 0 && (reinterpret_cast<uintptr_t>(gext) % ((uint64_t)k.vec * elem)) == 0) ? 1u : 0u;
   }
   p.n = c->N; p.stride = c->stride; p.j_base = c->j_base;
-  p.seed = c->seed; p.t = t; p.W = c->W; p.tp = tp;
+  p.seed = c->seed; p.W = c->W; p.tp = tp;
+  p.t = c->capturing ? t - c->capture_base : t;
+  p.t_dev = c->capturing ? c->sched : nullptr;
   p.warm_up_steps = c->warm_up_steps; p.identical_workers = c->identical ? 1u : 0u;
   p.worker_base = c->worker_base;
   p.eta = c->eta; p.eps = c->eps; p.sigma = c->sigma;
@@ -399,7 +412,9 @@ int launch_period(la_ctx* c, uint32_t h, bool post) {
   p.X = c->X; p.B2 = c->B2; p.Bs = c->Bs;
   p.a = c->pa; p.c = c->pc; p.s = c->has_s ? c->ps : nullptr;
   p.n = c->N; p.stride = c->stride; p.j_base = c->j_base;
-  p.seed = c->seed; p.t = c->t; p.W = c->W; p.tp = c->tp;
+  p.seed = c->seed; p.W = c->W; p.tp = c->tp;
+  p.t = c->capturing ? c->t - c->capture_base : c->t;
+  p.t_dev = c->capturing ? c->sched : nullptr;
   p.warm_up_steps = c->warm_up_steps; p.identical_workers = c->identical ? 1u : 0u;
   p.worker_base = c->worker_base;
   p.eta = c->eta; p.eps = c->eps; p.sigma = c->sigma;
@@ -546,6 +561,8 @@ void la_destroy(la_ctx* c) {
   for (auto*& m : c->ipc_opened) if (m) { cudaIpcCloseMemHandle(m); m = nullptr; }
   if (c->S) cudaFree(c->S);
   if (c->diag) cudaFree(c->diag);
+  if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
+  if (c->sched) cudaFree(c->sched);
   if (c->owns_arena && c->arena) cudaFree(c->arena);
   delete c;
 }
@@ -633,6 +650,18 @@ int la_set_rule(la_ctx* c, int rule) {
   return LA_OK;
 }
 
+int la_set_graph(la_ctx* c, int on) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (on && c->stream == nullptr) return fail(c, LA_ESTATE, "graph replay needs a context on a non-default stream (the legacy default stream cannot be captured)");
+  DeviceGuard guard(c->device);
+  if (on && !c->sched) {
+    cudaError_t e = cudaMalloc((void**)&c->sched, sizeof(uint64_t));
+    if (e != cudaSuccess) { c->sched = nullptr; cudaGetLastError(); return fail(c, LA_ENOMEM, "cudaMalloc failed: %s", cudaGetErrorString(e)); }
+  }
+  c->use_graph = on != 0;
+  return LA_OK;
+}
+
 int la_set_profiling(la_ctx* c, int on) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   DeviceGuard guard(c->device);
@@ -704,9 +733,81 @@ int la_sync(la_ctx* c) {
   return LA_OK;
 }
 
+static int run_steps(la_ctx* c, uint64_t T);
+
+// Capture one whole period (H iterations from t' = 0, exactly the launches run_steps would make)
+// into a CUDA graph.  The kernels take the step index as "offset within the period + *sched", so
+// the same graph serves every period; its last node advances *sched by H.
+static int ensure_period_graph(la_ctx* c) {
+  uint64_t key[8] = {(uint64_t)c->fusion | ((uint64_t)c->rule << 8) | ((uint64_t)c->grad_kind << 16) |
+                         ((uint64_t)c->bf16 << 24) | ((uint64_t)c->identical << 25) | ((uint64_t)c->has_s << 26),
+                     c->seed, (uint64_t)c->warm_up_steps | ((uint64_t)c->blocks_per_sm << 32),
+                     (uint64_t)c->worker_base | ((uint64_t)c->H << 32), 0, 0, 0, 1};
+  std::memcpy(&key[4], &c->sigma, sizeof(float));
+  std::memcpy(&key[5], &c->eta, sizeof(float));
+  std::memcpy(&key[6], &c->eps, sizeof(float));
+  if (c->graph_exec && std::memcmp(key, c->graph_key, sizeof key) == 0) return LA_OK;
+  if (c->graph_exec) { cudaGraphExecDestroy(c->graph_exec); c->graph_exec = nullptr; }
+  const uint64_t t0 = c->t, ns0 = c->nsync;
+  const uint32_t tp0 = c->tp;
+  const la_stats st0 = c->stats;
+  LA_CUDA(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+  c->capturing = true;
+  c->capture_base = c->t;
+  int rc = run_steps(c, c->H);
+  if (rc == LA_OK) {
+    la::la_counter_add<<<1, 1, 0, c->stream>>>(c->sched, (uint64_t)c->H);
+    if (cudaGetLastError() != cudaSuccess) rc = fail(c, LA_ECUDA, "launch of the counter node failed");
+  }
+  c->capturing = false;
+  cudaGraph_t graph = nullptr;
+  cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
+  // what one replay adds to the statistics; then undo the bookkeeping of the (unexecuted) capture
+  c->graph_delta = la_stats{};
+  c->graph_delta.launches_local = c->stats.launches_local - st0.launches_local;
+  c->graph_delta.launches_sync = c->stats.launches_sync - st0.launches_sync;
+  c->graph_delta.launches_fused = c->stats.launches_fused - st0.launches_fused;
+  c->graph_delta.launches_other = 1;
+  c->graph_delta.bytes_local = c->stats.bytes_local - st0.bytes_local;
+  c->graph_delta.bytes_sync = c->stats.bytes_sync - st0.bytes_sync;
+  c->graph_delta.bytes_fused = c->stats.bytes_fused - st0.bytes_fused;
+  c->stats = st0; c->t = t0; c->tp = tp0; c->nsync = ns0;
+  if (rc != LA_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+  if (e != cudaSuccess || !graph) { cudaGetLastError(); return fail(c, LA_ECUDA, "stream capture failed: %s", cudaGetErrorString(e)); }
+  e = cudaGraphInstantiate(&c->graph_exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (e != cudaSuccess) { c->graph_exec = nullptr; cudaGetLastError(); return fail(c, LA_ECUDA, "cudaGraphInstantiate failed: %s", cudaGetErrorString(e)); }
+  std::memcpy(c->graph_key, key, sizeof key);
+  return LA_OK;
+}
+
 int la_run(la_ctx* c, uint64_t T) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   DeviceGuard guard(c->device);
+  // Launch-bound regime (small N): replay whole periods from a captured graph.
+  if (c->use_graph && !c->profiling && c->rule != LA_RULE_ADAGRAD && c->fusion != LA_FUSE_SYNC_STEP && c->tp == 0 &&
+      c->H <= 4096u && T >= (uint64_t)c->H) {
+    int rc = ensure_period_graph(c);
+    if (rc) return rc;
+    const uint64_t reps = T / c->H;
+    la::la_counter_set<<<1, 1, 0, c->stream>>>(c->sched, c->t);
+    LA_CUDA(c, cudaGetLastError());
+    for (uint64_t k = 0; k < reps; ++k) LA_CUDA(c, cudaGraphLaunch(c->graph_exec, c->stream));
+    c->t += reps * c->H;
+    c->nsync += reps;
+    c->stats.launches_local += reps * c->graph_delta.launches_local;
+    c->stats.launches_sync += reps * c->graph_delta.launches_sync;
+    c->stats.launches_fused += reps * c->graph_delta.launches_fused;
+    c->stats.launches_other += reps * c->graph_delta.launches_other + 1;
+    c->stats.bytes_local += (double)reps * c->graph_delta.bytes_local;
+    c->stats.bytes_sync += (double)reps * c->graph_delta.bytes_sync;
+    c->stats.bytes_fused += (double)reps * c->graph_delta.bytes_fused;
+    T -= reps * c->H;
+  }
+  return run_steps(c, T);
+}
+
+static int run_steps(la_ctx* c, uint64_t T) {
   // Algorithm 3: for t in [T]: local step; if mod(t, H) == 0 (tracked as t' == H): synchronise.
   // `deferred` marks a synchronisation that is due but has been folded into the next step.
   if (c->rule == LA_RULE_ADAGRAD) {  // Algorithm 1: every iteration is one fully synchronous pass

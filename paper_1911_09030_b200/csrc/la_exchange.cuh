@@ -116,14 +116,14 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_step_export(const SweepPara
 
   __shared__ uint64_t keys[kMaxWorkers];
   if (kNeedsNoise) {
-    if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, p.t, p.identical_workers ? 0u : p.worker_base + threadIdx.x);
+    if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, step_index(p), p.identical_workers ? 0u : p.worker_base + threadIdx.x);
     __syncthreads();
   }
   const float eps2 = __fmul_rn(p.eps, p.eps);
   const float q = __fmul_rn(__uint2float_rn(p.tp), eps2);
   float eta_t = p.eta;
   if (p.warm_up_steps != 0u) {
-    const float ratio = __fdiv_rn(__ull2float_rn(p.t), __uint2float_rn(p.warm_up_steps));
+    const float ratio = __fdiv_rn(__ull2float_rn(step_index(p)), __uint2float_rn(p.warm_up_steps));
     eta_t = __fmul_rn(p.eta, fminf(1.0f, ratio));
   }
 
@@ -197,14 +197,14 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_import_step(const SweepPara
   const uint32_t W = (W_ > 0) ? (uint32_t)W_ : p.W;
   __shared__ uint64_t keys[kMaxWorkers];
   if (kNeedsNoise) {
-    if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, p.t, p.identical_workers ? 0u : p.worker_base + threadIdx.x);
+    if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, step_index(p), p.identical_workers ? 0u : p.worker_base + threadIdx.x);
     __syncthreads();
   }
   const float eps2 = __fmul_rn(p.eps, p.eps);
   const float q = __fmul_rn(__uint2float_rn(p.tp), eps2);  // p.tp == 1: first step of the period
   float eta_t = p.eta;
   if (p.warm_up_steps != 0u) {
-    const float ratio = __fdiv_rn(__ull2float_rn(p.t), __uint2float_rn(p.warm_up_steps));
+    const float ratio = __fdiv_rn(__ull2float_rn(step_index(p)), __uint2float_rn(p.warm_up_steps));
     eta_t = __fmul_rn(p.eta, fminf(1.0f, ratio));
   }
   const uint64_t ngroups = (p.n + (uint64_t)(V - 1)) / (uint64_t)V;

@@ -41,7 +41,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_period(const PeriodParams p
   if (kNeedsNoise) {
     for (uint32_t k = threadIdx.x; k < h * W; k += blockDim.x) {
       const uint32_t s = k / W, i = k - s * W;
-      keys[s][i] = step_worker_key(p.seed, p.t + 1u + s, p.identical_workers ? 0u : p.worker_base + i);
+      keys[s][i] = step_worker_key(p.seed, step_index(p) + 1u + s, p.identical_workers ? 0u : p.worker_base + i);
     }
   }
   if (threadIdx.x < h) {
@@ -50,7 +50,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_period(const PeriodParams p
     q_s[s] = __fmul_rn(__uint2float_rn(p.tp + 1u + s), eps2);  // t' eps^2 of step s
     float e = p.eta;
     if (p.warm_up_steps != 0u) {
-      const float ratio = __fdiv_rn(__ull2float_rn(p.t + 1u + s), __uint2float_rn(p.warm_up_steps));
+      const float ratio = __fdiv_rn(__ull2float_rn(step_index(p) + 1u + s), __uint2float_rn(p.warm_up_steps));
       e = __fmul_rn(p.eta, fminf(1.0f, ratio));
     }
     eta_s[s] = e;

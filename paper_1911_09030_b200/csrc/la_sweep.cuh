@@ -45,7 +45,9 @@ struct SweepParams {
   uint64_t stride;     // replica stride in floats (multiple of 64, >= N rounded up to 4)
   uint64_t j_base;     // global index of coordinate 0 (multiple of 4)
   uint64_t seed;
-  uint64_t t;          // 1-based global step index of the STEP part
+  uint64_t t;          // 1-based global step index of the STEP part ...
+  const uint64_t* t_dev;  // ... plus *t_dev when non-null: a device-resident step counter, so that a
+                          // captured CUDA graph of one period can be replayed without new arguments
   uint32_t W;
   uint32_t tp;         // t' of the STEP part (local steps since the last sync, incl. this one)
   uint32_t warm_up_steps;
@@ -53,6 +55,10 @@ struct SweepParams {
   uint32_t worker_base;  // global index of local replica 0 (sharding by worker); keys use worker_base + i
   float eta, eps, sigma;
 };
+
+__device__ __forceinline__ uint64_t step_index(const SweepParams& p) {
+  return p.t + (p.t_dev != nullptr ? *p.t_dev : 0ull);
+}
 
 constexpr int kMaxWorkers = 64;
 constexpr int kTreeDepth = 7;  // log2(kMaxWorkers) + 1 partial sums
@@ -326,7 +332,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
 
   __shared__ uint64_t keys[kMaxWorkers];
   if (kNeedsNoise) {
-    if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, p.t, p.identical_workers ? 0u : p.worker_base + threadIdx.x);
+    if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, step_index(p), p.identical_workers ? 0u : p.worker_base + threadIdx.x);
     __syncthreads();
   }
 
@@ -337,7 +343,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
     q = __fmul_rn(__uint2float_rn(p.tp), eps2);  // t' eps^2, the placeholder of Section 4.2
     eta_t = p.eta;
     if (p.warm_up_steps != 0u) {  // Section 6.2: eta_t = eta min(1, t / warm_up_steps)
-      const float ratio = __fdiv_rn(__ull2float_rn(p.t), __uint2float_rn(p.warm_up_steps));
+      const float ratio = __fdiv_rn(__ull2float_rn(step_index(p)), __uint2float_rn(p.warm_up_steps));
       eta_t = __fmul_rn(p.eta, fminf(1.0f, ratio));
     }
   }
@@ -460,13 +466,13 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_adagrad(const SweepParams p
   const uint32_t W = (W_ > 0) ? (uint32_t)W_ : p.W;
   __shared__ uint64_t keys[kMaxWorkers];
   if (kNeedsNoise) {
-    if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, p.t, p.identical_workers ? 0u : p.worker_base + threadIdx.x);
+    if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, step_index(p), p.identical_workers ? 0u : p.worker_base + threadIdx.x);
     __syncthreads();
   }
   const float eps2 = __fmul_rn(p.eps, p.eps);
   float eta_t = p.eta;
   if (p.warm_up_steps != 0u) {
-    const float ratio = __fdiv_rn(__ull2float_rn(p.t), __uint2float_rn(p.warm_up_steps));
+    const float ratio = __fdiv_rn(__ull2float_rn(step_index(p)), __uint2float_rn(p.warm_up_steps));
     eta_t = __fmul_rn(p.eta, fminf(1.0f, ratio));
   }
   const uint64_t ngroups = (p.n + (uint64_t)(V - 1)) / (uint64_t)V;

@@ -67,6 +67,7 @@ def lib() -> C.CDLL:
             "la_set_rule": [vp, i32],
             "la_set_launch_shape": [vp, i32],
             "la_set_profiling": [vp, i32],
+            "la_set_graph": [vp, i32],
             "la_local_step": [vp],
             "la_local_step_grads": [vp, vp, i32],
             "la_step_grads": [vp, vp, i32],
@@ -250,6 +251,9 @@ class LocalAdaAlter:
 
     def set_launch_shape(self, blocks_per_sm):
         self._ck(self.L.la_set_launch_shape(self.h, int(blocks_per_sm)))
+
+    def set_graph(self, on=True):
+        self._ck(self.L.la_set_graph(self.h, int(bool(on))))
 
     def set_profiling(self, on=True):
         self._ck(self.L.la_set_profiling(self.h, int(bool(on))))

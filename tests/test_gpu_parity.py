@@ -432,3 +432,46 @@ def test_diagnostics_objective_and_replica_spread():
     assert g.diagnostics()[1] == 0.0
     g.set_grad_noise(1, None)
     assert np.isnan(g.diagnostics()[0])
+
+
+@pytest.mark.parametrize("fusion", [0, 1, 3])
+@pytest.mark.parametrize("rule", [0, 1])
+def test_graph_replay_is_bitwise_and_counts_the_same(fusion, rule):
+    """la_set_graph: whole periods replayed from a captured CUDA graph (launch-bound sizes)."""
+    import torch
+    n, W, H = 6000, 4, 4
+    arr = _arrays(n, 17)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        g = la.LocalAdaAlter.with_torch_arena([n], W, 0.1, 1.0, H)
+        p = la.LocalAdaAlter.with_torch_arena([n], W, 0.1, 1.0, H)          # same, launched plainly
+        o = Oracle(n, W, 0.1, 1.0, H)
+        for ctx in (g, p):
+            ctx.set_grad_quadratic(5, arr["a"], arr["c"], 0.3)
+            ctx.set_warmup(7)
+            ctx.set_rule(rule)
+            ctx.set_fusion(fusion)
+        o.set_grad_quadratic(5, arr["a"], arr["c"], 0.3)
+        o.set_warmup(7)
+        o.set_rule(rule)
+        g.set_graph(True)
+        for T in (9, 3, 12, 2):                     # 9 = two periods + one step; then starts inside a period
+            g.run(T); p.run(T); o.run(T)
+            assert g.get_counters() == o.counters() == p.get_counters()
+        compare(g, o, W, TOL_RUN)
+        sg, sp = g.get_stats(), p.get_stats()
+        for k in ("launches_local", "launches_sync", "launches_fused", "bytes_local", "bytes_sync", "bytes_fused"):
+            assert sg[k] == sp[k], k
+        # a changed configuration rebuilds the graph
+        g.set_grad_noise(9, arr["s"]); o.set_grad_noise(9, arr["s"])
+        g.run(2); o.run(2)                          # finish the open period (t' = 2 -> 0)
+        g.run(8); o.run(8)
+        compare(g, o, W, TOL_RUN)
+        g.close(); p.close()
+
+
+def test_graph_replay_needs_a_capturable_stream():
+    g = la.LocalAdaAlter([64], 2, 0.1, 1.0, 2)      # legacy default stream
+    with pytest.raises(la.LocalAdaAlterError) as e:
+        g.set_graph(True)
+    assert e.value.code == la.LA_ESTATE
+    g.run(4)
