@@ -475,3 +475,59 @@ def test_graph_replay_needs_a_capturable_stream():
         g.set_graph(True)
     assert e.value.code == la.LA_ESTATE
     g.run(4)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_call_sequences_match_oracle(seed):
+    """Random interleavings of la_run / la_local_step / la_sync / fusion and launch-shape changes,
+    state round trips and rule changes at period boundaries, mirrored on the oracle."""
+    rng = np.random.default_rng(seed)
+    n = int(rng.integers(1, 5000))
+    W = int(rng.choice([1, 2, 3, 4, 8, 16, 6]))
+    H = int(rng.integers(1, 7))
+    arr = _arrays(n, seed)
+    grad = ["noise", "noise_scaled", "quadratic"][seed % 3]
+    g, o = make_pair(n, W, 0.05, 0.7, H, grad, seed=seed, arrays=arr, sigma=0.4, b0sq=0.5)
+    rule = 0
+    for _ in range(40):
+        op = rng.integers(0, 8)
+        if op <= 2:
+            T = int(rng.integers(0, 3 * H + 2))
+            g.run(T); o.run(T)
+        elif op == 3:
+            g.local_step(); o.local_step()
+            if rule == 0 and o.counters()[1] >= H and rng.random() < 0.5:
+                g.sync(); o.sync()
+        elif op == 4:
+            g.sync(); o.sync()
+        elif op == 5:
+            g.set_fusion(int(rng.integers(0, 4)))
+            g.set_launch_shape(int(rng.choice([0, 1, 7, 4096])))
+        elif op == 6 and o.counters()[1] == 0:
+            rule = int(rng.integers(0, 2))                       # Local AdaAlter <-> Local SGD
+            g.set_rule(rule); o.set_rule(rule)
+        elif op == 7:
+            i = int(rng.integers(0, W))
+            x, b2, bs = g.read_state(i)
+            g.write_state(i, x, b2, bs)                          # a checkpoint round trip changes nothing
+        assert g.get_counters() == o.counters()
+    compare(g, o, W, TOL_RUN)
+
+
+def test_two_contexts_on_two_streams_do_not_interfere():
+    import torch
+    n, W = 200003, 4
+    arr = _arrays(n, 2)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    with torch.cuda.stream(s1):
+        g1 = la.LocalAdaAlter.with_torch_arena([n], W, 0.1, 1.0, 3)
+    with torch.cuda.stream(s2):
+        g2 = la.LocalAdaAlter.with_torch_arena([n], W, 0.2, 0.5, 2)
+    g1.set_grad_quadratic(1, arr["a"], arr["c"], 0.3)
+    g2.set_grad_noise(2, arr["s"])
+    for _ in range(5):                                           # interleaved enqueueing
+        g1.run(3); g2.run(4)
+    o1 = Oracle(n, W, 0.1, 1.0, 3); o1.set_grad_quadratic(1, arr["a"], arr["c"], 0.3); o1.run(15)
+    o2 = Oracle(n, W, 0.2, 0.5, 2); o2.set_grad_noise(2, arr["s"]); o2.run(20)
+    compare(g1, o1, W, TOL_RUN)
+    compare(g2, o2, W, TOL_RUN)
