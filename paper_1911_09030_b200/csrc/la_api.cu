@@ -24,6 +24,9 @@ SweepKernel lookup_sweep_w2(int, int, bool, bool, bool, bool);
 SweepKernel lookup_sweep_w4(int, int, bool, bool, bool, bool);
 SweepKernel lookup_sweep_w8(int, int, bool, bool, bool, bool);
 SweepKernel lookup_sweep_w16(int, int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w3(int, int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w6(int, int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w12(int, int, bool, bool, bool, bool);
 
 SweepKernel lookup_sweep(int W, int rule, int gm, bool bf16, bool pre, bool step, bool post) {
   switch (W) {
@@ -32,6 +35,9 @@ SweepKernel lookup_sweep(int W, int rule, int gm, bool bf16, bool pre, bool step
     case 4: return lookup_sweep_w4(rule, gm, bf16, pre, step, post);
     case 8: return lookup_sweep_w8(rule, gm, bf16, pre, step, post);
     case 16: return lookup_sweep_w16(rule, gm, bf16, pre, step, post);
+    case 3: return lookup_sweep_w3(rule, gm, bf16, pre, step, post);
+    case 6: return lookup_sweep_w6(rule, gm, bf16, pre, step, post);
+    case 12: return lookup_sweep_w12(rule, gm, bf16, pre, step, post);
     default: return lookup_sweep_w0(rule, gm, bf16, pre, step, post);
   }
 }
@@ -42,6 +48,9 @@ PeriodKernel lookup_period_w2(int, bool, bool);
 PeriodKernel lookup_period_w4(int, bool, bool);
 PeriodKernel lookup_period_w8(int, bool, bool);
 PeriodKernel lookup_period_w16(int, bool, bool);
+PeriodKernel lookup_period_w3(int, bool, bool);
+PeriodKernel lookup_period_w6(int, bool, bool);
+PeriodKernel lookup_period_w12(int, bool, bool);
 
 PeriodKernel lookup_period(int W, int gm, bool bf16, bool post) {
   switch (W) {
@@ -50,6 +59,9 @@ PeriodKernel lookup_period(int W, int gm, bool bf16, bool post) {
     case 4: return lookup_period_w4(gm, bf16, post);
     case 8: return lookup_period_w8(gm, bf16, post);
     case 16: return lookup_period_w16(gm, bf16, post);
+    case 3: return lookup_period_w3(gm, bf16, post);
+    case 6: return lookup_period_w6(gm, bf16, post);
+    case 12: return lookup_period_w12(gm, bf16, post);
     default: return lookup_period_w0(gm, bf16, post);
   }
 }
@@ -58,6 +70,7 @@ PeriodKernel lookup_period(int W, int gm, bool bf16, bool post) {
   StepExportFn lookup_step_export_w##w(int, bool);       \
   ImportStepFn lookup_import_step_w##w(int, bool);
 LA_DECL_XCH(0) LA_DECL_XCH(1) LA_DECL_XCH(2) LA_DECL_XCH(4) LA_DECL_XCH(8) LA_DECL_XCH(16)
+LA_DECL_XCH(3) LA_DECL_XCH(6) LA_DECL_XCH(12)
 #undef LA_DECL_XCH
 
 StepExportFn lookup_step_export(int W, int gm, bool bf16) {
@@ -67,6 +80,9 @@ StepExportFn lookup_step_export(int W, int gm, bool bf16) {
     case 4: return lookup_step_export_w4(gm, bf16);
     case 8: return lookup_step_export_w8(gm, bf16);
     case 16: return lookup_step_export_w16(gm, bf16);
+    case 3: return lookup_step_export_w3(gm, bf16);
+    case 6: return lookup_step_export_w6(gm, bf16);
+    case 12: return lookup_step_export_w12(gm, bf16);
     default: return lookup_step_export_w0(gm, bf16);
   }
 }
@@ -77,6 +93,9 @@ ImportStepFn lookup_import_step(int W, int gm, bool bf16) {
     case 4: return lookup_import_step_w4(gm, bf16);
     case 8: return lookup_import_step_w8(gm, bf16);
     case 16: return lookup_import_step_w16(gm, bf16);
+    case 3: return lookup_import_step_w3(gm, bf16);
+    case 6: return lookup_import_step_w6(gm, bf16);
+    case 12: return lookup_import_step_w12(gm, bf16);
     default: return lookup_import_step_w0(gm, bf16);
   }
 }
@@ -87,6 +106,9 @@ ExchangeFn lookup_export_w2();
 ExchangeFn lookup_export_w4();
 ExchangeFn lookup_export_w8();
 ExchangeFn lookup_export_w16();
+ExchangeFn lookup_export_w3();
+ExchangeFn lookup_export_w6();
+ExchangeFn lookup_export_w12();
 
 ExchangeFn lookup_export(int W) {
   switch (W) {
@@ -95,6 +117,9 @@ ExchangeFn lookup_export(int W) {
     case 4: return lookup_export_w4();
     case 8: return lookup_export_w8();
     case 16: return lookup_export_w16();
+    case 3: return lookup_export_w3();
+    case 6: return lookup_export_w6();
+    case 12: return lookup_export_w12();
     default: return lookup_export_w0();
   }
 }

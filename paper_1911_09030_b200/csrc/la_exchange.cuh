@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(LA_BLOCK) la_export_sums(const ExchangeParams 
   for (uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < ngroups; grp += nthreads) {
     const uint64_t off = grp * V;
     uint64_t addr = x_base + off * sizeof(float);
-    PairTree<V> tree;
+    typename TreeFor<W_, V>::type tree;
 #pragma unroll kOuterUnroll
     for (uint32_t i0 = 0; i0 < W; i0 += CH) {
       ReplicaChunk<V, CH> ch;
@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(LA_BLOCK) la_combine_sums(const ExchangeParams
   const uint64_t nthreads = (uint64_t)gridDim.x * blockDim.x;
   for (uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < ngroups; grp += nthreads) {
     const uint64_t off = p.slice_lo + grp * V;
-    PairTree<V> tree;
+    PairTreeDyn<V> tree;
     for (uint32_t r = 0; r < p.world; ++r) {
       // plain loads; for r != rank these are peer loads over NVLink.  Not the streaming
       // (evict-first) flavour: a peer's line is fetched once and not re-read.
@@ -153,7 +153,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_step_export(const SweepPara
     const CoordInputs<V> in = in_next;
     const uint64_t ctr0 = kGoldenGamma * (((p.j_base + off) >> 1) + 1u);
     const Vec<V> r = step_size<V>(in.bs, q, eta_t);
-    PairTree<V> tree;
+    typename TreeFor<W_, V>::type tree;
 #pragma unroll kOuterUnroll
     for (uint32_t i0 = 0; i0 < W; i0 += CH) {
       ReplicaChunk<V, CH> cur = nxt;

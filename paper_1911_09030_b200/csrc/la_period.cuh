@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_period(const PeriodParams p
     // it unrolled the kernel body (W x 8 copies of the gradient source) overflowed the
     // instruction cache and a fifth of the issue slots went to instruction-fetch stalls.
     for (uint32_t s = 0; s < h; ++s) r_s[s][threadIdx.x] = step_size<V>(in.bs, q_s[s], eta_s[s]);
-    PairTree<V> tree;
+    typename TreeFor<W_, V>::type tree;
 
 #pragma unroll kOuterUnroll
     for (uint32_t i0 = 0; i0 < W; i0 += CH) {

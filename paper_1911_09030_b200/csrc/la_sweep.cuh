@@ -18,6 +18,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <cstdint>
+#include <type_traits>
 
 #include "grad_source.cuh"
 
@@ -171,6 +172,62 @@ struct PairTree {
       if (ACC) b[ACC ? sp - 1 : 0] = add(b[ACC ? sp - 1 : 0], b[ACC ? sp : 0]);
     }
   }
+};
+
+// The same tree when the number of workers is only known at run time.  One slot per level, like
+// the digits of a binary counter: pushing worker number n walks up the levels, merging (older
+// partial sum on the left) while bit L of n is set and parking the carry in the first clear
+// level.  Every slot index is a compile-time constant (the run-time part is predication), so the
+// partial sums stay in registers; a stack with a run-time top would live in local memory.
+template <int V, bool ACC = true>
+struct PairTreeDyn {
+  Vec<V> x[kTreeDepth], b[ACC ? kTreeDepth : 1];
+  uint32_t n = 0;
+  __device__ __forceinline__ void push(uint32_t, const Vec<V>& vx, const Vec<V>& vb) {
+    Vec<V> cx = vx, cb = vb;
+    bool placed = false;
+#pragma unroll
+    for (int L = 0; L < kTreeDepth; ++L) {
+      if (!placed) {
+        if ((n >> L) & 1u) {
+          cx = add(x[L], cx);
+          if (ACC) cb = add(b[ACC ? L : 0], cb);
+        } else {
+          x[L] = cx;
+          if (ACC) b[ACC ? L : 0] = cb;
+          placed = true;
+        }
+      }
+    }
+    ++n;
+  }
+  // Leaves the total in x[0], b[0]: the occupied levels are merged from the lowest up, each
+  // higher (older) level on the left.
+  __device__ __forceinline__ void finish() {
+    Vec<V> ax = x[0], ab = b[0];
+    bool have = false;
+#pragma unroll
+    for (int L = 0; L < kTreeDepth; ++L) {
+      if ((n >> L) & 1u) {
+        if (have) {
+          ax = add(x[L], ax);
+          if (ACC) ab = add(b[ACC ? L : 0], ab);
+        } else {
+          ax = x[L];
+          if (ACC) ab = b[ACC ? L : 0];
+          have = true;
+        }
+      }
+    }
+    x[0] = ax;
+    if (ACC) b[0] = ab;
+  }
+};
+
+// Static worker count: the stack form (constant indices after unrolling); otherwise the counter form.
+template <int W_, int V, bool ACC = true>
+struct TreeFor {
+  using type = typename std::conditional<(W_ > 0), PairTree<V, ACC>, PairTreeDyn<V, ACC>>::type;
 };
 
 // Worker-independent data of one coordinate group: the stale accumulator and the problem arrays.
@@ -387,7 +444,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
     Vec<V> r;
     if (kLoadsBs) r = step_size<V>(in.bs, q, eta_t);
     if (!ACC) r = splat<V>(eta_t);
-    PairTree<V, ACC> tree;
+    typename TreeFor<W_, V, ACC>::type tree;
 
 #pragma unroll kOuterUnroll
     for (uint32_t i0 = 0; i0 < W; i0 += CH) {
@@ -484,7 +541,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_adagrad(const SweepParams p
     Vec<V> x = ld_stream<V>(p.X + off);
     Vec<V> b = ld_stream<V>(p.B2 + off);
     const uint64_t ctr0 = kGoldenGamma * (((p.j_base + off) >> 1) + 1u);
-    PairTree<V, false> tree;
+    typename TreeFor<W_, V, false>::type tree;
 #pragma unroll kOuterUnroll
     for (uint32_t i = 0; i < W; ++i) {
       const Vec<V> g = gradient<GM, false, V>(p, in, x, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
