@@ -531,3 +531,20 @@ def test_two_contexts_on_two_streams_do_not_interfere():
     o2 = Oracle(n, W, 0.2, 0.5, 2); o2.set_grad_noise(2, arr["s"]); o2.run(20)
     compare(g1, o1, W, TOL_RUN)
     compare(g2, o2, W, TOL_RUN)
+
+
+@pytest.mark.parametrize("fusion", [1, 3])
+def test_paper_hyperparameters(fusion):
+    """The settings of the paper's experiments (Section 6): eps = 1, b0 = 1, eta = 0.5 with 600
+    warm-up steps, 8 workers, H = 4 (the period the paper recommends)."""
+    n, W, H, T = 20000, 8, 4, 24
+    arr = _arrays(n, 44)
+    g, o = make_pair(n, W, 0.5, 1.0, H, "quadratic", seed=6, arrays=arr, sigma=1.0, b0sq=1.0, warmup=600,
+                     fusion=fusion)
+    g.run(1); o.run(1)
+    compare(g, o, W, TOL_STEP)
+    g.run(T - 1); o.run(T - 1)
+    compare(g, o, W, TOL_RUN)
+    x, _, _ = o.read(0)
+    xd, _, _ = o.read_shadow(0)
+    assert np.max(np.abs(x - xd)) < 1e-5          # fp32 path tracks the literal fp64 formulas
