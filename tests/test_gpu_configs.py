@@ -120,3 +120,34 @@ def test_beyond_32_bit_indexing():
                 assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), (lo, i)
         assert g.get_counters() == o.counters()
     g.close()
+
+
+def test_config2_four_million_coordinates_full_run():
+    """Configuration 2, full W and T, on 2^22 coordinates (64 blocks of 2^16 spread evenly over the
+    vector), the oracle running one block per host thread."""
+    import os
+    from concurrent.futures import ThreadPoolExecutor
+    wl = workloads.config("c2")
+    arr = wl.arrays()
+    g = _make_gpu(wl, arr, wl.H, la.LA_FUSE_STEP_SYNC)
+    g.run(wl.T)
+    blocks = [(k * (wl.N // 64), k * (wl.N // 64) + (1 << 16)) for k in range(64)]
+    import threading
+    ctx_lock = threading.Lock()                      # a context serves one caller thread at a time
+
+    def check(rng):
+        lo, hi = rng
+        o = _make_oracle(wl, arr, wl.H, lo, hi)
+        o.run(wl.T)
+        bad = 0
+        for i in range(wl.W):
+            with ctx_lock:
+                got = g.read_range(i, lo, hi - lo)
+            for a, b in zip(got, o.read(i)):
+                bad += int(np.count_nonzero(a.view(np.uint32) != b.view(np.uint32)))
+        return bad
+
+    with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as ex:
+        mismatches = sum(ex.map(check, blocks))
+    assert mismatches == 0
+    g.close()
