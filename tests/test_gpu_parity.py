@@ -548,3 +548,16 @@ def test_paper_hyperparameters(fusion):
     x, _, _ = o.read(0)
     xd, _, _ = o.read_shadow(0)
     assert np.max(np.abs(x - xd)) < 1e-5          # fp32 path tracks the literal fp64 formulas
+
+
+@pytest.mark.parametrize("W", [24, 48])
+def test_run_time_worker_counts_over_many_blocks(W):
+    """Worker counts without a dedicated kernel, on enough coordinates for several blocks per SM
+    and a ragged tail, through every fusion mode."""
+    n, H, T = 150001, 3, 7
+    arr = _arrays(n, W)
+    for fusion in (0, 1, 2, 3):
+        g, o = make_pair(n, W, 0.05, 1.0, H, "noise_scaled", seed=W, arrays=arr, fusion=fusion)
+        g.run(T); o.run(T)
+        compare(g, o, W, TOL_RUN)
+        g.close()
