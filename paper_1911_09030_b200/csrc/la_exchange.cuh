@@ -50,7 +50,7 @@ __global__ void __launch_bounds__(LA_BLOCK) la_export_sums(const ExchangeParams 
       load_chunk<V, CH>(ch, addr, b_delta, stride_bytes, W, i0);
 #pragma unroll
       for (int k = 0; k < CH; ++k)
-        if (i0 + k < W) tree.push(i0 + k, ch.x[k], ch.b[k]);
+        if (i0 + k < W) tree.push_in_chunk(i0 + k, k, i0 + CH <= W, ch.x[k], ch.b[k]);
     }
     tree.finish();
     st_stream<V>(out + off, tree.x[0]);
@@ -178,7 +178,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_step_export(const SweepPara
           const Vec<V> g = kExternal ? gcur.g[kExternal ? k : 0]
                                      : gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
           apply<V>(r, g, cur.x[k], cur.b[k]);
-          tree.push(i, cur.x[k], cur.b[k]);
+          tree.push_in_chunk(i, k, i0 + CH <= W, cur.x[k], cur.b[k]);
         }
     }
     tree.finish();

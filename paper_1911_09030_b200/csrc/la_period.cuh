@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_period(const PeriodParams p
             apply<V>(r_s[s][threadIdx.x], g, cur.x[k], cur.b[k]);
           }
           if (POST) {
-            tree.push(i, cur.x[k], cur.b[k]);
+            tree.push_in_chunk(i, k, i0 + CH <= W, cur.x[k], cur.b[k]);
           } else {
             store_replica<V>(st_addr, b_delta, stride_bytes, cur.x[k], cur.b[k]);
           }

@@ -165,6 +165,10 @@ struct PairTree {
       if (ACC) b[ACC ? sp - 1 : 0] = add(b[ACC ? sp - 1 : 0], b[ACC ? sp : 0]);
     }
   }
+  // position k within a chunk of replicas is irrelevant here (see PairTreeDyn)
+  __device__ __forceinline__ void push_in_chunk(uint32_t i, int, bool, const Vec<V>& vx, const Vec<V>& vb) {
+    push(i, vx, vb);
+  }
   __device__ __forceinline__ void finish() {
     while (sp > 1) {
       --sp;
@@ -201,6 +205,50 @@ struct PairTreeDyn {
     }
     ++n;
   }
+  // Push of a partial sum that already covers 2^LOG consecutive workers starting at a multiple
+  // of 2^LOG: the walk up the levels simply starts at level LOG.
+  template <int LOG>
+  __device__ __forceinline__ void push_block(const Vec<V>& vx, const Vec<V>& vb) {
+    Vec<V> cx = vx, cb = vb;
+    bool placed = false;
+#pragma unroll
+    for (int L = LOG; L < kTreeDepth; ++L) {
+      if (!placed) {
+        if ((n >> L) & 1u) {
+          cx = add(x[L], cx);
+          if (ACC) cb = add(b[ACC ? L : 0], cb);
+        } else {
+          x[L] = cx;
+          if (ACC) b[ACC ? L : 0] = cb;
+          placed = true;
+        }
+      }
+    }
+    n += 1u << LOG;
+  }
+  // Replica i = i0 + k of a chunk of four that starts at a multiple of four.  When the chunk is
+  // complete its members are first summed as (v0 + v1) + (v2 + v3) — the bottom two levels of
+  // the same tree — with compile-time positions, and enter the counter as one block: a quarter
+  // of the run-time level walks.
+  __device__ __forceinline__ void push_in_chunk(uint32_t i, int k, bool chunk_complete, const Vec<V>& vx,
+                                                const Vec<V>& vb) {
+    if (!chunk_complete) {
+      push(i, vx, vb);
+    } else if (k == 0) {
+      px0 = vx; pb0 = vb;
+    } else if (k == 1) {
+      px0 = add(px0, vx);
+      if (ACC) pb0 = add(pb0, vb);
+    } else if (k == 2) {
+      px1 = vx; pb1 = vb;
+    } else {
+      px1 = add(px1, vx);
+      if (ACC) pb1 = add(pb1, vb);
+      push_block<2>(add(px0, px1), ACC ? add(pb0, pb1) : pb0);
+    }
+  }
+  Vec<V> px0, px1, pb0, pb1;
+
   // Leaves the total in x[0], b[0]: the occupied levels are merged from the lowest up, each
   // higher (older) level on the left.
   __device__ __forceinline__ void finish() {
@@ -468,13 +516,13 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
         if (i0 + k < W) {
           const uint32_t i = i0 + k;
           if (PRE) {
-            tree.push(i, cur.x[k], cur.b[k]);
+            tree.push_in_chunk(i, k, i0 + CH <= W, cur.x[k], cur.b[k]);
           } else {
             const Vec<V> g = kExternal ? gcur.g[kExternal ? k : 0]
                                        : gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
             apply<V, ACC>(r, g, cur.x[k], cur.b[k]);
             if (POST) {
-              tree.push(i, cur.x[k], cur.b[k]);
+              tree.push_in_chunk(i, k, i0 + CH <= W, cur.x[k], cur.b[k]);
             } else {
               store_replica<V, ACC>(st_addr, b_delta, stride_bytes, cur.x[k], cur.b[k]);
             }
