@@ -119,7 +119,8 @@ int la_set_identical_workers(la_ctx* ctx, int on);
 /* Warm-up of Section 6.2: eta_t = eta * min(1, t / warm_up_steps); 0 switches it off. */
 int la_set_warmup(la_ctx* ctx, uint32_t warm_up_steps);
 /* Baseline update rules of the paper in the same sweep (LA_RULE_*): Local SGD (Algorithm 2) and
- * Distributed AdaGrad (Algorithm 1), for fp32 generated gradients.  Only legal while t' == 0.
+ * Distributed AdaGrad (Algorithm 1), for fp32 generated gradients and for supplied gradient
+ * tables (la_local_step_grads, la_step_grads).  Only legal while t' == 0.
  * AdaGrad keeps ONE shared iterate (all workers see x_{t-1}); W only sets how many gradients are
  * averaged per step; la_read_state returns that iterate for any worker, la_sync is LA_ESTATE,
  * and n_sync counts one gradient exchange per iteration. */

@@ -352,6 +352,8 @@ double pass_bytes(const la_ctx* c, bool pre, bool step, bool post, int gm) {
   const double n = (double)c->N, W = (double)c->W;
   if (c->rule == LA_RULE_ADAGRAD) {                 // one shared x, B2: read + write, Bs written
     double b = 20.0 * n;
+    if (gm == la::kGradExternalF32) b += 4.0 * W * n;
+    if (gm == la::kGradExternalBF16) b += 2.0 * W * n;
     if (gm == la::kGradQuadratic) b += 8.0 * n;
     if (gm == la::kGradNoiseScaled || (gm == la::kGradConstant && c->has_s)) b += 4.0 * n;
     return b;
@@ -359,6 +361,8 @@ double pass_bytes(const la_ctx* c, bool pre, bool step, bool post, int gm) {
   if (c->rule == LA_RULE_LOCAL_SGD) {               // X only: read + write
     double b = 8.0 * W * n;
     if (step) {
+      if (gm == la::kGradExternalF32) b += 4.0 * W * n;
+      if (gm == la::kGradExternalBF16) b += 2.0 * W * n;
       if (gm == la::kGradQuadratic) b += 8.0 * n;
       if (gm == la::kGradNoiseScaled || (gm == la::kGradConstant && c->has_s)) b += 4.0 * n;
     }
@@ -718,12 +722,13 @@ int la_local_step_grads(la_ctx* c, const void* g_dev, int dtype) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   if (!g_dev) return fail(c, LA_EINVAL, "g_dev is NULL");
   if (dtype != LA_F32 && dtype != LA_BF16) return fail(c, LA_EINVAL, "dtype must be LA_F32 or LA_BF16");
-  if (c->rule != LA_RULE_ADAALTER) return fail(c, LA_ESTATE, "supplied gradients are implemented for Local AdaAlter only");
   DeviceGuard guard(c->device);
   int rc = launch_sweep(c, false, true, false, c->t + 1, c->tp + 1,
                         dtype == LA_F32 ? la::kGradExternalF32 : la::kGradExternalBF16, g_dev);
   if (rc) return rc;
-  c->t += 1; c->tp += 1;
+  c->t += 1;
+  if (c->rule == LA_RULE_ADAGRAD) c->nsync += 1;
+  else c->tp += 1;
   return LA_OK;
 }
 
@@ -731,7 +736,7 @@ int la_step_grads(la_ctx* c, const void* g_dev, int dtype) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   if (!g_dev) return fail(c, LA_EINVAL, "g_dev is NULL");
   if (dtype != LA_F32 && dtype != LA_BF16) return fail(c, LA_EINVAL, "dtype must be LA_F32 or LA_BF16");
-  if (c->rule != LA_RULE_ADAALTER) return fail(c, LA_ESTATE, "supplied gradients are implemented for Local AdaAlter only");
+  if (c->rule == LA_RULE_ADAGRAD) return la_local_step_grads(c, g_dev, dtype);  // Algorithm 1: one pass is the whole iteration
   DeviceGuard guard(c->device);
   const int gm = dtype == LA_F32 ? la::kGradExternalF32 : la::kGradExternalBF16;
   const bool closes = (c->tp + 1 == c->H);

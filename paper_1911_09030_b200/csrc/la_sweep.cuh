@@ -567,6 +567,8 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
 template <int W_, int V, int GM, int MINB>
 __global__ void __launch_bounds__(LA_BLOCK, MINB) la_adagrad(const SweepParams p) {
   constexpr bool kNeedsNoise = (GM == kGradNoise || GM == kGradNoiseScaled || GM == kGradQuadratic);
+  constexpr bool kExternal = (GM == kGradExternalF32 || GM == kGradExternalBF16);
+  constexpr uint64_t kGradElem = (GM == kGradExternalBF16) ? 2 : 4;
   constexpr int kOuterUnroll = (W_ > 0) ? kMaxWorkers : 1;
   const uint32_t W = (W_ > 0) ? (uint32_t)W_ : p.W;
   __shared__ uint64_t keys[kMaxWorkers];
@@ -590,9 +592,17 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_adagrad(const SweepParams p
     Vec<V> b = ld_stream<V>(p.B2 + off);
     const uint64_t ctr0 = kGoldenGamma * (((p.j_base + off) >> 1) + 1u);
     typename TreeFor<W_, V, false>::type tree;
+    uint64_t g_addr = reinterpret_cast<uint64_t>(p.gext) + off * kGradElem;  // supplied gradients, row by row
 #pragma unroll kOuterUnroll
     for (uint32_t i = 0; i < W; ++i) {
-      const Vec<V> g = gradient<GM, false, V>(p, in, x, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
+      Vec<V> g;
+      if (kExternal) {
+        GradChunk<V, 1> gc;
+        load_grads<GM, V, 1>(gc, p, g_addr, p.n * kGradElem, W, i, off);
+        g = gc.g[0];
+      } else {
+        g = gradient<GM, false, V>(p, in, x, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
+      }
       tree.push(i, g, g);
     }
     tree.finish();

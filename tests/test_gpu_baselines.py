@@ -81,3 +81,30 @@ def test_three_rules_on_one_problem_behave_as_the_paper_describes():
         g.set_rule(rule)
         g.run(T)
         assert f(g.read_state(0)[0]) < 0.2 * f0
+
+
+@pytest.mark.parametrize("rule", [la.LA_RULE_LOCAL_SGD, la.LA_RULE_ADAGRAD])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("W,n", [(4, 4098), (3, 777), (8, 70000)])
+def test_baselines_with_supplied_gradients(rule, dtype, W, n):
+    """The trainer-facing call (la_step_grads) under the two baseline rules."""
+    import torch
+    H, T = 3, 7
+    rng = np.random.default_rng(n + W)
+    g = la.LocalAdaAlter([n], W, 0.2, 0.5, H)
+    g.set_rule(rule)
+    g.set_fusion(la.LA_FUSE_STEP_SYNC)
+    o = Oracle(n, W, 0.2, 0.5, H)
+    o.set_rule(rule)
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    code = la.LA_F32 if dtype == "f32" else la.LA_BF16
+    for t in range(T):
+        G = torch.from_numpy(rng.standard_normal((W, n)).astype(np.float32)).to(tdt)
+        Gd = G.cuda()
+        g.step_grads(Gd.data_ptr(), code)
+        o.local_step(G.float().numpy())
+        if rule == la.LA_RULE_LOCAL_SGD and o.counters()[1] == H:
+            o.sync()
+        g.sync_stream()
+        assert g.get_counters() == o.counters()
+    compare(g, o, W, 1e-5)
