@@ -31,8 +31,8 @@ FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from
 # the ncu capture summarised in profiles/), valid only for the kernel sources they were taken on.
-KERNEL_HASH_AT_CAPTURE = "9eb400846fb9ddf5"
-NCU_TRAFFIC_BYTES = {"c2": 2.2239e9}
+KERNEL_HASH_AT_CAPTURE = "f7182c402edd33c4"
+NCU_TRAFFIC_BYTES = {"c2": 2.2240e9}
 
 
 def kernel_source_hash():
