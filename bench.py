@@ -173,7 +173,7 @@ def run_reference(args, wl):
 # lanes = 18 944 lane-instructions per clock; lane-instructions per worker*param update from the
 # ncu capture summarised in profiles/ (smsp__inst_executed.sum x 32 / updates per launch).
 LANE_INSTR_PER_CLOCK = 148 * 4 * 32
-PERIOD_LANE_INSTR_PER_UPDATE = {"c2": 50.4}
+PERIOD_LANE_INSTR_PER_UPDATE = {"c2": 50.5}
 
 
 def alu_roofline(period, wl, clocks):
