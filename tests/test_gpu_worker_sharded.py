@@ -1,7 +1,7 @@
 """Sharding by worker on the GPU: the three-phase synchronisation (export / combine / import)
-against the single-context kernels and the oracle.  One GPU is available, so several ranks are
-emulated as several contexts of one process on one stream (their kernels never wait for each
-other; the host orders the phases)."""
+against the single-context kernels and the oracle.  Several ranks are emulated as several
+contexts of one process on one GPU and one stream (their kernels never wait for each other;
+the host orders the phases)."""
 import numpy as np
 import pytest
 

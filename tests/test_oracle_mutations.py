@@ -72,7 +72,7 @@ def _run_one(name):
 
 @pytest.fixture(scope="module")
 def mutation_results():
-    """All mutants are built and judged concurrently (one pytest child each)."""
+    """All mutants are built and evaluated concurrently (one pytest child each)."""
     from concurrent.futures import ThreadPoolExecutor
     with ThreadPoolExecutor(max_workers=max(2, (os.cpu_count() or 2))) as ex:
         return {name: (rc, out) for name, rc, out in ex.map(_run_one, sorted(MUTATIONS))}
