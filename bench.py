@@ -1,13 +1,19 @@
 #!/usr/bin/env python
 """Benchmark of the Local AdaAlter hot path (Algorithm 3 of arXiv 1911.09030) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5] [--impl ours|reference]
 
 A "step" is one `la_run(T)` of the chosen configuration: T iterations of Algorithm 3 for all
-W workers over all N coordinates, including the synchronisations that fall in it.  Prints ONE
-JSON line.  With N > 1 GPUs (torchrun) each rank runs the same configuration on its own
-coordinate range (coordinates never interact, so there is no data-path collective): weak
-scaling.  `--impl reference` times the CPU oracle, as it stands, on a bounded sample.
+W workers over all N coordinates, including the synchronisations that fall in it.  The default
+workload is the largest single-GPU configuration (c5: 200 ragged tensors, 4e8 coordinates, four
+workers, bf16-rounded gradients, 13.4 GiB of state).  Prints ONE JSON line: the whole-run rate,
+per-kernel durations and HBM roofline fractions of the local step (K1), the stand-alone
+synchronisation (K2) and both fusions (K3, K4), the temporal-blocking mode, the end-to-end rate
+with host buffers, the CPU oracle on the host cores, and — on one GPU — configuration 2 and the
+synchronisation-period sweep of configuration 4.  With N > 1 GPUs (torchrun) each rank runs the
+same configuration on its own coordinate range (coordinates never interact, so there is no
+data-path collective): weak scaling.  `--impl reference` times the CPU oracle, as it stands, on
+a bounded sample.
 """
 from __future__ import annotations
 
@@ -29,23 +35,26 @@ METRIC = "worker_param_updates_per_sec"
 UNIT = "worker*param updates/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum from
-# the ncu capture summarised in profiles/), valid only for the kernel sources they were taken on.
+# Figures taken from the ncu captures summarised in profiles/, valid only for the kernel sources
+# they were taken on (KERNEL_HASH_AT_CAPTURE):
+#   NCU_TRAFFIC_BYTES             dram__bytes_read.sum + dram__bytes_write.sum per K1 launch
+#   PERIOD_LANE_INSTR_PER_UPDATE  smsp__inst_executed.sum x 32 / updates per la_period launch
 KERNEL_HASH_AT_CAPTURE = "f7182c402edd33c4"
 NCU_TRAFFIC_BYTES = {"c2": 2.2240e9}
+PERIOD_LANE_INSTR_PER_UPDATE = {"c2": 50.5}
 
 
 def kernel_source_hash():
-    """Hash of what defines the la_sweep kernels: the two headers and the tuning macros."""
+    """Hash of what defines the kernels: the device headers and the tuning macros."""
     import hashlib
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_1911_09030_b200", "csrc")
-    for name in ("grad_source.cuh", "la_sweep.cuh"):
+    for name in ("grad_source.cuh", "la_sweep.cuh", "la_period.cuh", "la_exchange.cuh"):
         with open(os.path.join(d, name), "rb") as fh:
             h.update(fh.read())
     with open(os.path.join(d, "la_sweep_inst.inc")) as fh:
         for line in fh:
-            if line.startswith("#define LA_VEC") or line.startswith("#define LA_MINB"):
+            if line.startswith("#define LA_"):
                 h.update(line.encode())
     return h.hexdigest()[:16]
 
@@ -61,7 +70,8 @@ def measured_peak():
 
 # --------------------------------------------------------------------------- clocks
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs (read-only)."""
+    """Samples nvidia-smi clocks and throttle reasons for the whole invocation (read-only);
+    `window(t0, t1)` summarises the samples that fell inside one timed region."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -85,16 +95,20 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append((time.time(), line.strip()))
 
-    def stop(self, t0: float, t1: float):
+    def stop(self):
         if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return
         time.sleep(0.15)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=2)
         except Exception:
             self.proc.kill()
-        rows = [l for (ts, l) in self.lines if t0 <= ts <= t1 + 0.2] or [l for _, l in self.lines]
+
+    def window(self, t0: float, t1: float):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        rows = [l for (ts, l) in list(self.lines) if t0 <= ts <= t1 + 0.2]
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for l in rows:
@@ -113,15 +127,19 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------- oracle leg
-def oracle_rate(wl, n_slice: int, threads: int = 1, T=None):
-    """worker*param updates/s of the CPU oracle on the first n_slice coordinates at full W and T."""
+ORACLE_UPDATES_PER_CORE_S = 4.5e7     # order of magnitude, only used to bound the sample size
+
+
+def oracle_rate(wl, j0: int, n_slice: int, threads: int = 1, T=None):
+    """worker*param updates/s of the CPU oracle on coordinates [j0, j0 + n_slice) at full W and T,
+    the slice cut into `threads` contiguous ranges, one per host thread."""
     from concurrent.futures import ThreadPoolExecutor
     from oracle.oracle import Oracle
     T = wl.T if T is None else T
     per = n_slice // threads
     jobs = []
     for k in range(threads):
-        lo = k * per
+        lo = j0 + k * per
         arr = wl.arrays(lo, per)
         o = Oracle(per, wl.W, wl.eta, wl.eps, wl.H, wl.b0sq, j_base=lo)
         if wl.grad == "quadratic":
@@ -143,17 +161,41 @@ def oracle_rate(wl, n_slice: int, threads: int = 1, T=None):
     return per * threads * wl.W * T / dt, dt
 
 
+def bounded_slice(wl, want: int, seconds: float) -> int:
+    """Largest power of two <= want whose single-core oracle run stays near `seconds`."""
+    n = min(want, wl.N)
+    while n > 1024 and n * wl.W * wl.T / ORACLE_UPDATES_PER_CORE_S > seconds:
+        n //= 2
+    return n
+
+
+def cpu_baseline(wl):
+    """The oracle as it stands on a contiguous slice of the workload (2^22 coordinates when one
+    core finishes that in about half a minute) at full W and T: one core, then all cores."""
+    n_slice = bounded_slice(wl, 1 << 22, 40.0)
+    v, dt = oracle_rate(wl, 0, n_slice)
+    cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt,
+           "sample": f"contiguous slice of {n_slice} coordinates [0, {n_slice}) of {wl.name} at full W={wl.W}, T={wl.T}"}
+    ncores = os.cpu_count() or 1
+    if ncores > 1:      # the same loop on disjoint coordinate ranges, one per host core
+        th = min(ncores, 32)
+        va, dta = oracle_rate(wl, 0, n_slice // th * th, threads=th)
+        cpu["all_cores"] = {"value": va, "cores": th, "seconds": dta,
+                            "sample": f"the same slice cut into {th} contiguous ranges, one host thread each"}
+    return cpu
+
+
 def run_reference(args, wl):
     """The reference arm: the oracle (plain single-threaded C++), timed as it stands."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    n_slice = min(wl.N, 1 << 14)
+    n_slice = bounded_slice(wl, 1 << 18, 1.5)
     for _ in range(args.warmup):
-        oracle_rate(wl, 1024)
+        oracle_rate(wl, 0, 1024)
     rates, t_all = [], 0.0
     for _ in range(args.steps):
-        r, dt = oracle_rate(wl, n_slice)
+        r, dt = oracle_rate(wl, 0, n_slice)
         rates.append(r); t_all += dt
     value = float(np.mean(rates))
     sample = f"first {n_slice} coordinates of {wl.name} at full W={wl.W}, T={wl.T}, per step"
@@ -171,22 +213,26 @@ def run_reference(args, wl):
 
 # Issue-slot roofline of the temporal-blocking kernel (la_period): 148 SMs x 4 schedulers x 32
 # lanes = 18 944 lane-instructions per clock; lane-instructions per worker*param update from the
-# ncu capture summarised in profiles/ (smsp__inst_executed.sum x 32 / updates per launch).
+# ncu captures summarised in profiles/ (smsp__inst_executed.sum x 32 / updates per launch), valid
+# only while the kernel sources hash to the captured version.
 LANE_INSTR_PER_CLOCK = 148 * 4 * 32
-PERIOD_LANE_INSTR_PER_UPDATE = {"c2": 50.5}
 
 
 def alu_roofline(period, wl, clocks):
     if period is None:
         return None
     out = dict(period)
-    ipu = PERIOD_LANE_INSTR_PER_UPDATE.get(wl.name)
+    ipu = PERIOD_LANE_INSTR_PER_UPDATE.get(wl.name) if kernel_source_hash() == KERNEL_HASH_AT_CAPTURE else None
     max_mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+    sm_mhz = (clocks or {}).get("sm_mhz")
     peak = LANE_INSTR_PER_CLOCK * max_mhz * 1e6 / 1e12          # T lane-instr/s at the maximum SM clock
+    out["clocks"] = clocks
     if ipu:
-        ach = period["value"] * ipu / 1e12
+        ach = period["value"] / period["n_gpus"] * ipu / 1e12
         out["roofline"] = {"bound": "alu", "achieved": ach, "peak": peak, "unit": "T lane-instr/s",
-                           "frac": ach / peak, "lane_instr_per_update": ipu, "traffic": None}
+                           "frac": ach / peak, "lane_instr_per_update": ipu, "traffic": None,
+                           "peak_at_sampled_clock": (LANE_INSTR_PER_CLOCK * sm_mhz * 1e6 / 1e12) if sm_mhz else None,
+                           "frac_at_sampled_clock": (ach / (LANE_INSTR_PER_CLOCK * sm_mhz * 1e6 / 1e12)) if sm_mhz else None}
     return out
 
 
@@ -199,10 +245,105 @@ def workload_config(wl, args):
 
 
 # --------------------------------------------------------------------------- CUDA leg
+KERNEL_NAMES = {"local": "K1 local step", "sync": "K2 sync", "step_sync": "K3 step+sync",
+                "sync_step": "K4 sync+next step", "period": "temporal blocking"}
+
+
+def per_kernel(stats, peak, leg):
+    """Per-kernel figures from the library's event-timed statistics of one profiled leg."""
+    out = {}
+    for cls in KERNEL_NAMES:
+        n = stats[f"launches_{cls}"]
+        ms_all = stats[f"ms_{cls}"]
+        if not n or ms_all <= 0:
+            continue
+        ms = ms_all / n
+        b = stats[f"bytes_{cls}"] / n
+        gbs = b / (ms * 1e-3) / 1e9
+        out[cls] = {"kernel": KERNEL_NAMES[cls], "launches": int(n), "ms_per_launch": ms, "bytes_per_launch": b,
+                    "GBps": gbs, "frac": gbs / peak, "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
+                    "ms_total": ms_all, "leg": leg}
+    return out
+
+
+class Job:
+    """One configuration resident on this rank's GPU."""
+
+    def __init__(self, la, wl, j_base=0, pinned=False):
+        import torch
+        self.la, self.wl, self.torch = la, wl, torch
+        arr = wl.arrays()        # same per-coordinate inputs on every rank; noise differs through j_base
+        self.ctx = la.LocalAdaAlter.with_torch_arena(wl.sizes, wl.W, wl.eta, wl.eps, wl.H, b0sq=wl.b0sq, j_base=j_base)
+        self.stream = torch.cuda.current_stream()
+        self.pinned = None
+        if pinned:
+            self.pinned = {k: torch.from_numpy(v).pin_memory() for k, v in arr.items()}
+            self.x0_pin = torch.zeros(wl.N, dtype=torch.float32).pin_memory()
+            self.out_pin = {k: torch.empty(wl.N, dtype=torch.float32).pin_memory() for k in ("x", "b2", "bs")}
+            self.h2d = 4 * wl.N * (1 + len(arr))
+            self.d2h = 4 * wl.N * 3
+            self.upload()
+        else:
+            c = self.ctx
+            if wl.grad == "quadratic":
+                c.set_grad_quadratic(wl.noise_seed, arr["a"], arr["c"], wl.sigma)
+            elif wl.grad == "noise_scaled":
+                c.set_grad_noise(wl.noise_seed, arr["s"])
+            else:
+                c.set_grad_noise(wl.noise_seed, None)
+        if wl.bf16_grads:
+            self.ctx.set_grad_dtype(la.LA_BF16)
+
+    def upload(self):
+        """The step's inputs from pinned host memory, through the C-ABI (enqueued on the stream)."""
+        c, wl, p = self.ctx, self.wl, self.pinned
+        c._ck(c.L.la_set_init(c.h, self.x0_pin.data_ptr(), float(wl.b0sq)))
+        if wl.grad == "quadratic":
+            c._ck(c.L.la_set_grad_quadratic(c.h, wl.noise_seed, p["a"].data_ptr(), p["c"].data_ptr(), float(wl.sigma)))
+        elif wl.grad == "noise_scaled":
+            c._ck(c.L.la_set_grad_noise(c.h, wl.noise_seed, p["s"].data_ptr()))
+        else:
+            c._ck(c.L.la_set_grad_noise(c.h, wl.noise_seed, None))
+
+    def download(self):
+        c, o = self.ctx, self.out_pin
+        c._ck(c.L.la_read_state(c.h, 0, o["x"].data_ptr(), o["b2"].data_ptr(), o["bs"].data_ptr()))
+
+    def timed(self, fusion, steps, warmup, barrier, profiling=False, H=None, T=None):
+        """`steps` x la_run(T) on the device; returns (ms per step, library statistics, wall window)."""
+        torch, c = self.torch, self.ctx
+        T = self.wl.T if T is None else T
+        c.set_fusion(fusion)
+        for _ in range(warmup):
+            c.run(T)
+        barrier()
+        c.get_stats(reset=True)
+        c.set_profiling(profiling)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        w0 = time.time()
+        e0.record(self.stream)
+        for _ in range(steps):
+            c.run(T)
+        e1.record(self.stream)
+        barrier()
+        w1 = time.time()
+        ms = e0.elapsed_time(e1) / steps
+        stats = c.get_stats(reset=True)
+        c.set_profiling(False)
+        return ms, stats, (w0, w1)
+
+    def close(self):
+        self.ctx.close()
+        self.pinned = self.out_pin = self.x0_pin = None
+        self.torch.cuda.empty_cache()
+
+
 def run_ours(args, wl):
     import torch
     import torch.distributed as dist
     from paper_1911_09030_b200 import local_adaalter as la
+    from paper_1911_09030_b200 import sharding, workloads
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -212,162 +353,171 @@ def run_ours(args, wl):
     if use_dist:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dd = dist if use_dist else None
 
     def barrier():
         if use_dist:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # this rank's coordinate range: the same configuration, shifted (weak scaling)
-    from paper_1911_09030_b200 import sharding
-    j_base = sharding.weak_scaling_base(wl.N, rank)
-    arr = wl.arrays()            # same per-coordinate inputs on every rank; noise differs through j_base
-    stream = torch.cuda.current_stream()
-    ctx = la.LocalAdaAlter.with_torch_arena(wl.sizes, wl.W, wl.eta, wl.eps, wl.H, b0sq=wl.b0sq, j_base=j_base)
-
-    pinned = {k: torch.from_numpy(v).pin_memory() for k, v in arr.items()}
-    x0_pin = torch.zeros(wl.N, dtype=torch.float32).pin_memory()
-    out_pin = {k: torch.empty(wl.N, dtype=torch.float32).pin_memory() for k in ("x", "b2", "bs")}
-
-    def upload():
-        ctx._ck(ctx.L.la_set_init(ctx.h, x0_pin.data_ptr(), float(wl.b0sq)))
-        if wl.grad == "quadratic":
-            ctx._ck(ctx.L.la_set_grad_quadratic(ctx.h, wl.noise_seed, pinned["a"].data_ptr(),
-                                                 pinned["c"].data_ptr(), float(wl.sigma)))
-        elif wl.grad == "noise_scaled":
-            ctx._ck(ctx.L.la_set_grad_noise(ctx.h, wl.noise_seed, pinned["s"].data_ptr()))
-        else:
-            ctx._ck(ctx.L.la_set_grad_noise(ctx.h, wl.noise_seed, None))
-    h2d = 4 * wl.N * (1 + len(arr))
-    d2h = 4 * wl.N * 3
-
-    upload()
-    if wl.bf16_grads:
-        ctx.set_grad_dtype(la.LA_BF16)
-    ctx.set_fusion(args.fusion)
-    if args.blocks_per_sm:
-        ctx.set_launch_shape(args.blocks_per_sm)
-
-    # ---- device-resident timing -----------------------------------------------------------
-    for _ in range(args.warmup):
-        ctx.run(wl.T)
-    barrier()
-    ctx.get_stats(reset=True)
-    ctx.set_profiling(True)
     vis = [v for v in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if v]
     sampler = ClockSampler(vis[local_rank] if local_rank < len(vis) else str(local_rank))
     if rank == 0:
         sampler.start()
-        time.sleep(0.25)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    t_wall0 = time.time()
-    e0.record(stream)
-    for _ in range(args.steps):
-        ctx.run(wl.T)
-    e1.record(stream)
-    barrier()
-    t_wall1 = time.time()
-    ms_total = e0.elapsed_time(e1)
-    stats = ctx.get_stats(reset=True)
-    ctx.set_profiling(False)
-    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+
+    # this rank's coordinate range: the same configuration, shifted (weak scaling)
+    job = Job(la, wl, j_base=sharding.weak_scaling_base(wl.N, rank), pinned=True)
+    if args.blocks_per_sm:
+        job.ctx.set_launch_shape(args.blocks_per_sm)
+    units = wl.W * wl.N * wl.T * world
+    peak, peak_kind = measured_peak()
+
+    # ---- headline: device-resident, per-launch profiling off --------------------------------
+    ms_step, stats_main, win_main = job.timed(args.fusion, args.steps, args.warmup, barrier)
+    ms_step = sharding.max_over_ranks(ms_step, dd)
+    launches_main = int(stats_main["launches_local"] + stats_main["launches_sync"] + stats_main["launches_fused"])
+    bytes_main = stats_main["bytes_local"] + stats_main["bytes_sync"] + stats_main["bytes_fused"]
+
+    # ---- the same run again with CUDA events around every launch: per-kernel durations -------
+    kernels = {}
+    _, st, _ = job.timed(args.fusion, args.steps, 1, barrier, profiling=True)
+    kernels.update(per_kernel(st, peak, f"la_run, fusion {args.fusion}, {args.steps} steps"))
+    short = max(1, min(args.steps, 3))
+    if not args.main_only:
+        for fusion in (la.LA_FUSE_NONE, la.LA_FUSE_STEP_SYNC, la.LA_FUSE_SYNC_STEP):
+            if fusion == args.fusion:
+                continue
+            _, st, _ = job.timed(fusion, short, 1, barrier, profiling=True)
+            for k, v in per_kernel(st, peak, f"la_run, fusion {fusion}, {short} steps").items():
+                kernels.setdefault(k, v)
+    kernels.pop("period", None)
 
     # ---- the same job with temporal blocking (LA_FUSE_PERIOD): issue-bound instead of HBM-bound
     period = None
     if args.fusion != la.LA_FUSE_PERIOD and not args.no_period:
-        ctx.set_fusion(la.LA_FUSE_PERIOD)
-        for _ in range(2):
-            ctx.run(wl.T)
-        barrier()
-        ctx.get_stats(reset=True)
-        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        p0.record(stream)
-        for _ in range(args.steps):
-            ctx.run(wl.T)
-        p1.record(stream)
-        barrier()
-        pst = ctx.get_stats(reset=True)
-        pms = sharding.max_over_ranks(p0.elapsed_time(p1) / args.steps, dist if use_dist else None)
-        period = {"ms_per_step": pms, "value": wl.W * wl.N * wl.T * world / (pms * 1e-3), "unit": UNIT,
-                  "launches_per_step": pst["launches_fused"] // args.steps,
-                  "hbm_GBps": pst["bytes_fused"] / args.steps / (pms * 1e-3) / 1e9}
-        ctx.set_fusion(args.fusion)
+        psteps = max(1, min(args.steps, 5))
+        pms, pst, pwin = job.timed(la.LA_FUSE_PERIOD, psteps, 2, barrier)
+        pms = sharding.max_over_ranks(pms, dd)
+        period = {"ms_per_step": pms, "steps": psteps, "value": units / (pms * 1e-3), "unit": UNIT, "n_gpus": world,
+                  "launches_per_step": int(pst["launches_fused"]) // psteps,
+                  "hbm_GBps": pst["bytes_fused"] / psteps / (pms * 1e-3) / 1e9}
+        period = alu_roofline(period, wl, sampler.window(*pwin) if rank == 0 else None)
 
     # ---- end to end through the C-ABI with host buffers -------------------------------------
+    job.ctx.set_fusion(args.fusion)
+
     def e2e_step():
-        upload()
-        ctx.run(wl.T)
-        ctx._ck(ctx.L.la_read_state(ctx.h, 0, out_pin["x"].data_ptr(), out_pin["b2"].data_ptr(),
-                                    out_pin["bs"].data_ptr()))
+        job.upload()
+        job.ctx.run(wl.T)
+        job.download()                           # la_read_state synchronises the stream
     e2e_step()
     barrier()
-    t0 = time.perf_counter()
     e2e_steps = max(1, min(args.steps, 3))
+    t0 = time.perf_counter()
     for _ in range(e2e_steps):
-        e2e_step()                               # la_read_state synchronises the stream
+        e2e_step()
     barrier()
-    e2e_ms = 1e3 * (time.perf_counter() - t0) / e2e_steps
+    e2e_ms = sharding.max_over_ranks(1e3 * (time.perf_counter() - t0) / e2e_steps, dd)
+    h2d, d2h = job.h2d, job.d2h
+    job.close()
 
-    ms_total = sharding.max_over_ranks(ms_total, dist if use_dist else None)
-    e2e_ms = sharding.max_over_ranks(e2e_ms, dist if use_dist else None)
-    ms_per_step = ms_total / args.steps
-    units = wl.W * wl.N * wl.T * world
-    value = units / (ms_per_step * 1e-3)
+    # ---- the other bandwidth-bound configurations, on one GPU only ---------------------------
+    extras = {}
+    if world == 1 and not args.main_only:
+        if wl.name != "c2":
+            extras["c2"] = side_config(la, workloads.config("c2"), peak, barrier, sampler)
+        extras["c4_sync_period_sweep"] = sync_period_sweep(la, workloads.config("c4"), peak, barrier)
 
     if rank == 0:
-        peak, peak_kind = measured_peak()
-        launches = {k: stats[k] for k in ("launches_local", "launches_sync", "launches_fused")}
-        n_local = max(1, stats["launches_local"])
-        ms_local = stats["ms_local"] / n_local
-        bytes_local = stats["bytes_local"] / n_local
-        achieved = bytes_local / (ms_local * 1e-3) / 1e9 if ms_local > 0 else None
-        roofline = {
-            "bound": "hbm", "kernel": "la_sweep<STEP> (K1 local step)", "achieved": achieved, "peak": peak,
-            "peak_kind": peak_kind, "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
-            "traffic": (NCU_TRAFFIC_BYTES.get(wl.name) if kernel_source_hash() == KERNEL_HASH_AT_CAPTURE
-                        and args.H is None and args.N is None else None),
-            "frac_of_nominal_8TBps": (achieved / NOMINAL_HBM_GBS) if achieved else None,
-            "bytes_per_launch": bytes_local, "ms_per_launch": ms_local,
-            "bytes_per_update": bytes_local / (wl.W * wl.N),
-        }
-        per_class = {}
-        for cls in ("local", "sync", "fused"):
-            n = stats[f"launches_{cls}"]
-            if n:
-                ms = stats[f"ms_{cls}"] / n
-                per_class[cls] = {"launches": n, "ms_per_launch": ms,
-                                  "GBps": stats[f"bytes_{cls}"] / n / (ms * 1e-3) / 1e9 if ms > 0 else None,
-                                  "share_of_device_time": None}
-        tot = sum(stats[f"ms_{c}"] for c in ("local", "sync", "fused"))
-        for cls in per_class:
-            per_class[cls]["share_of_device_time"] = stats[f"ms_{cls}"] / tot if tot > 0 else None
+        sampler.stop()
+        clocks = sampler.window(*win_main)
+        k1 = kernels.get("local")
+        roofline = {"bound": "hbm", "kernel": "la_sweep<STEP> (K1 local step)", "achieved": None, "peak": peak,
+                    "peak_kind": peak_kind, "unit": "GB/s", "frac": None, "traffic": None}
+        if k1:
+            roofline.update({
+                "achieved": k1["GBps"], "frac": k1["frac"], "frac_of_nominal_8TBps": k1["frac_of_nominal_8TBps"],
+                "bytes_per_launch": k1["bytes_per_launch"], "ms_per_launch": k1["ms_per_launch"],
+                "bytes_per_update": k1["bytes_per_launch"] / (wl.W * wl.N), "launches": k1["launches"],
+                "timed": "CUDA events around every launch on the launching stream, in a repeat of the timed "
+                         "region with the library's per-launch profiling on (the headline value is timed with it off)",
+                "traffic": (NCU_TRAFFIC_BYTES.get(wl.name) if kernel_source_hash() == KERNEL_HASH_AT_CAPTURE
+                            and args.H is None and args.N is None else None)})
+        for cls, key in (("sync", "sync"), ("step_sync", "step_sync"), ("sync_step", "sync_step")):
+            k = kernels.get(cls)
+            if k:
+                roofline[key] = {"kernel": k["kernel"], "achieved": k["GBps"], "peak": peak, "unit": "GB/s",
+                                 "frac": k["frac"], "bytes_per_launch": k["bytes_per_launch"],
+                                 "ms_per_launch": k["ms_per_launch"], "launches": k["launches"]}
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
-            n_slice = min(wl.N, 1 << 16)
-            v, dt = oracle_rate(wl, n_slice)
-            cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt,
-                   "sample": f"first {n_slice} coordinates of {wl.name} at full W={wl.W}, T={wl.T}"}
-            ncores = os.cpu_count() or 1
-            if ncores > 1:      # the same loop on disjoint coordinate ranges, one per host core
-                va, dta = oracle_rate(wl, n_slice * min(ncores, 16) // 2, threads=min(ncores, 16))
-                cpu["all_cores"] = {"value": va, "cores": min(ncores, 16), "seconds": dta}
+            cpu = cpu_baseline(wl)
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "metric": METRIC, "value": units / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(wl, args),
             "clocks": clocks,
             "e2e": {"value": units / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
-            "gpu_launches": int(sum(launches.values())),
-            "roofline": roofline, "cpu_baseline": cpu, "kernels": per_class,
-            "temporal_blocking": alu_roofline(period, wl, clocks),
-            "hbm_GBps_whole_step": (stats["bytes_local"] + stats["bytes_sync"] + stats["bytes_fused"]) / (ms_total * 1e-3) / 1e9,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps},
+            "gpu_launches": launches_main,
+            "roofline": roofline, "cpu_baseline": cpu, "kernels": kernels,
+            "temporal_blocking": period,
+            "hbm_GBps_whole_step": bytes_main / args.steps / (ms_step * 1e-3) / 1e9,
         }
+        line.update(extras)
         print(json.dumps(line), flush=True)
-    ctx.close()
     if use_dist:
         dist.destroy_process_group()
+
+
+def side_config(la, wl, peak, barrier, sampler, steps=3):
+    """A further configuration in the same invocation: whole-run rate, K1/K3 figures, temporal blocking."""
+    job = Job(la, wl)
+    ms, _, _ = job.timed(la.LA_FUSE_STEP_SYNC, steps, 3, barrier)
+    _, st, _ = job.timed(la.LA_FUSE_STEP_SYNC, steps, 1, barrier, profiling=True)
+    units = wl.W * wl.N * wl.T
+    out = {"workload": workload_config(wl, None)["workload"], "steps": steps, "ms_per_step": ms,
+           "value": units / (ms * 1e-3), "unit": UNIT,
+           "kernels": per_kernel(st, peak, f"la_run, fusion 1, {steps} steps")}
+    pms, pst, pwin = job.timed(la.LA_FUSE_PERIOD, steps, 2, barrier)
+    period = {"ms_per_step": pms, "steps": steps, "value": units / (pms * 1e-3), "unit": UNIT, "n_gpus": 1,
+              "launches_per_step": int(pst["launches_fused"]) // steps,
+              "hbm_GBps": pst["bytes_fused"] / steps / (pms * 1e-3) / 1e9}
+    out["temporal_blocking"] = alu_roofline(period, wl, sampler.window(*pwin))
+    job.close()
+    return out
+
+
+def sync_period_sweep(la, wl, peak, barrier):
+    """Configuration 4: for every synchronisation period H, one full la_run(T) unfused (K1 + K2),
+    with the step fused into its synchronisation (K3) and with the synchronisation folded into the
+    next step (K4); share of device time spent synchronising.  The single-GPU analogue of the
+    2/H communication claim of Section 4.2."""
+    import copy
+    rows = []
+    for H in wl.H_sweep:
+        w = copy.copy(wl)
+        w.H = H
+        job = Job(la, w)
+        for fusion in (la.LA_FUSE_NONE, la.LA_FUSE_STEP_SYNC, la.LA_FUSE_SYNC_STEP):
+            job.ctx.set_fusion(fusion)
+            job.ctx.run(2 * H if 2 * H < w.T else w.T)      # warm-up: two periods
+            ms, st, _ = job.timed(fusion, 1, 0, barrier, profiling=True)
+            ker = per_kernel(st, peak, f"H={H}, fusion {fusion}")
+            tot = sum(st[f"ms_{c}"] for c in ("local", "sync", "fused"))
+            ms_k1 = ker["local"]["ms_per_launch"] if "local" in ker else None
+            sync_ms = st["ms_sync"]
+            if ms_k1 is not None:   # a fused pass is charged its excess over a plain local step
+                for c in ("step_sync", "sync_step"):
+                    if c in ker:
+                        sync_ms += st[f"launches_{c}"] * max(0.0, ker[c]["ms_per_launch"] - ms_k1)
+            rows.append({"H": H, "fusion": fusion, "T": w.T, "ms_per_run": ms,
+                         "value": w.W * w.N * w.T / (ms * 1e-3),
+                         "sync_share_of_device_time": sync_ms / tot if tot > 0 else None,
+                         "GBps": {c: round(v["GBps"], 1) for c, v in ker.items()},
+                         "launches": {c: v["launches"] for c, v in ker.items()}})
+        job.close()
+    return {"workload": workload_config(wl, None)["workload"].split(", H=")[0], "unit": UNIT, "rows": rows}
 
 
 def run_report(args):
@@ -514,7 +664,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--workload", default="c5", help="c1..c5; default: the largest single-GPU configuration")
     ap.add_argument("--H", type=int, default=None, help="override the synchronisation period")
     ap.add_argument("--T", type=int, default=None, help="override iterations per step")
     ap.add_argument("--N", type=int, default=None, help="override the size (one flat tensor), e.g. for small ncu captures")
@@ -522,6 +672,8 @@ def main():
     ap.add_argument("--blocks-per-sm", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-period", action="store_true", help="skip the extra temporal-blocking measurement")
+    ap.add_argument("--main-only", action="store_true",
+                    help="only the chosen workload in its fusion mode (no other fusion legs, no c2 / c4 extras)")
     ap.add_argument("--report", action="store_true", help="all configurations + the H sweep (not the JSON line)")
     ap.add_argument("--report-out", default=None)
     ap.add_argument("--tradeoff", action="store_true", help="quality/time against H on a noisy quadratic (table)")

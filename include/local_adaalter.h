@@ -79,10 +79,17 @@ typedef struct la_config {
 typedef struct la_stats {
   uint64_t launches_local;  /* K1: local step (gradient + update + accumulate), Algorithm 3 body */
   uint64_t launches_sync;   /* K2: stand-alone synchronisation */
-  uint64_t launches_fused;  /* K3/K4: a local step and a synchronisation in one pass */
+  uint64_t launches_fused;  /* every pass that holds a step AND a synchronisation, or several steps */
   uint64_t launches_other;  /* fills, scatter/gather of state */
   double ms_local, ms_sync, ms_fused; /* device time per class; only while profiling is on */
   double bytes_local, bytes_sync, bytes_fused; /* algorithmic HBM bytes issued per class */
+  /* the fused class split by kernel (exchange-fused steps of the by-worker path are in
+   * launches_fused only) */
+  uint64_t launches_step_sync; /* K3: step t'=H and its synchronisation */
+  uint64_t launches_sync_step; /* K4: synchronisation folded into the step t'=1 that follows */
+  uint64_t launches_period;    /* temporal blocking: several local steps (and the closing sync) */
+  double ms_step_sync, ms_sync_step, ms_period;
+  double bytes_step_sync, bytes_sync_step, bytes_period;
 } la_stats;
 
 /* ---- creation / destruction ------------------------------------------------
@@ -212,7 +219,9 @@ int la_diagnostics(la_ctx* ctx, double* objective, double* replica_spread);
  * that of worker worker_base + i.  W_total = 0 returns to the unsharded numbering. */
 int la_set_worker_range(la_ctx* ctx, uint32_t worker_base, uint32_t W_total);
 /* Allocate the exchange buffer (freed by la_destroy) and fix this context's rank.  If no worker
- * range was set: worker_base = rank * W, W_total = world * W. */
+ * range was set: worker_base = rank * W, W_total = world * W.  With world > 1 the local worker
+ * count W must be a power of two (LA_EINVAL otherwise): only then is "local tree, then tree over
+ * ranks" the adjacent-pair tree over all workers. */
 int la_comm_create(la_ctx* ctx, uint32_t rank, uint32_t world);
 /* Device pointer and size of the exchange buffer (2 * stride floats). */
 int la_comm_buffer(la_ctx* ctx, void** dev_ptr, uint64_t* bytes);
@@ -260,7 +269,11 @@ int la_stream_sync(la_ctx* ctx);
  *   b2_mean_dev      by (float)W — the same bits la_sync would put into every replica
  *   stream           a cudaStream_t (NULL = default); the work is only enqueued
  * The first call on a device looks up the array's device address (cudaGetSymbolAddress) with
- * that device current; make that first call outside any stream capture.  All calls share the
+ * that device current; make that first call outside any stream capture.  Under CUDA's default
+ * lazy module loading that first call is also when the driver sets the 8 MiB aside on that
+ * device (not when the library is loaded), so make it during start-up, before your own
+ * allocator takes what is left of the GPU, or run with CUDA_MODULE_LOADING=EAGER.  If it fails
+ * the call returns LA_ECUDA, leaves no sticky CUDA error behind and may simply be repeated.  All calls share the
  * one array: it is fully rewritten for [0, n) by each call (nothing needs to start at zero, and
  * it keeps the last call's sums afterwards), so two calls that overlap on the GPU — different
  * streams, or different threads — race; run them in stream order. */

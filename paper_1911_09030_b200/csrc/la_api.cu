@@ -138,6 +138,22 @@ __global__ void la_fill(float* X, float* B2, float* Bs, const float* x0, float b
   }
 }
 
+// Copies replica 0's x and B^2 into replicas 1..W-1 (Algorithm 1 keeps one iterate that every
+// worker holds; the AdaGrad kernel stores it once, and this materialises the other copies when
+// a per-worker view is needed again).
+__global__ void la_broadcast_replica0(float* X, float* B2, uint64_t stride, uint32_t W) {
+  const uint64_t nthreads = (uint64_t)gridDim.x * blockDim.x;
+  const uint64_t nvec = stride / 4;  // stride is a multiple of 64 floats
+  for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < nvec; j += nthreads) {
+    const float4 x = reinterpret_cast<const float4*>(X)[j];
+    const float4 b = reinterpret_cast<const float4*>(B2)[j];
+    for (uint32_t i = 1; i < W; ++i) {
+      reinterpret_cast<float4*>(X + (uint64_t)i * stride)[j] = x;
+      reinterpret_cast<float4*>(B2 + (uint64_t)i * stride)[j] = b;
+    }
+  }
+}
+
 // Device-resident step counter used by captured graphs (see la_set_graph).
 __global__ void la_counter_set(uint64_t* ctr, uint64_t v) { *ctr = v; }
 __global__ void la_counter_add(uint64_t* ctr, uint64_t v) { *ctr += v; }
@@ -196,7 +212,9 @@ namespace {
 thread_local std::string g_create_error;
 constexpr uint64_t kExchangeVecHost = la::kExchangeVec;
 
-enum KernelClass { kClassLocal = 0, kClassSync = 1, kClassFused = 2, kClassOther = 3 };
+// kClassStepSync, kClassSyncStep and kClassPeriod are also counted in the aggregate "fused" class.
+enum KernelClass { kClassLocal = 0, kClassSync = 1, kClassFused = 2, kClassOther = 3,
+                   kClassStepSync = 4, kClassSyncStep = 5, kClassPeriod = 6 };
 
 struct EventPair {
   cudaEvent_t a, b;
@@ -217,6 +235,7 @@ struct la_ctx {
   uint64_t seed = 0;
   int fusion = LA_FUSE_NONE;
   int rule = LA_RULE_ADAALTER;
+  bool shared_iterate = false;  // AdaGrad steps ran: replica 0 holds x_t, B^2_t; replicas 1..W-1 are stale
   bool profiling = false;
   int device = 0;
   cudaStream_t stream = nullptr;
@@ -321,7 +340,10 @@ int drain_events(la_ctx* c) {
     LA_CUDA(c, cudaEventElapsedTime(&ms, p.a, p.b));
     if (p.cls == kClassLocal) c->stats.ms_local += ms;
     else if (p.cls == kClassSync) c->stats.ms_sync += ms;
-    else if (p.cls == kClassFused) c->stats.ms_fused += ms;
+    else if (p.cls != kClassOther) c->stats.ms_fused += ms;
+    if (p.cls == kClassStepSync) c->stats.ms_step_sync += ms;
+    else if (p.cls == kClassSyncStep) c->stats.ms_sync_step += ms;
+    else if (p.cls == kClassPeriod) c->stats.ms_period += ms;
     c->pool.push_back(p);
   }
   c->pending.clear();
@@ -412,7 +434,7 @@ int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t
   const int bps = c->blocks_per_sm > 0 ? c->blocks_per_sm : (step ? 96 : 4096);
   const uint64_t cap = (uint64_t)c->num_sms * (uint64_t)bps;
   if (blocks > cap) blocks = cap;
-  const int cls = (step && (pre || post)) ? kClassFused : (step ? kClassLocal : kClassSync);
+  const int cls = !step ? kClassSync : (post ? kClassStepSync : (pre ? kClassSyncStep : kClassLocal));
   EventPair ep{};
   if (c->profiling) {
     int rc = begin_timed(c, cls, &ep);
@@ -427,7 +449,11 @@ int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t
   const double bytes = pass_bytes(c, pre, step, post, gm);
   if (cls == kClassLocal) { c->stats.launches_local++; c->stats.bytes_local += bytes; }
   else if (cls == kClassSync) { c->stats.launches_sync++; c->stats.bytes_sync += bytes; }
-  else { c->stats.launches_fused++; c->stats.bytes_fused += bytes; }
+  else {
+    c->stats.launches_fused++; c->stats.bytes_fused += bytes;
+    if (cls == kClassStepSync) { c->stats.launches_step_sync++; c->stats.bytes_step_sync += bytes; }
+    else { c->stats.launches_sync_step++; c->stats.bytes_sync_step += bytes; }
+  }
   return LA_OK;
 }
 
@@ -458,7 +484,7 @@ int launch_period(la_ctx* c, uint32_t h, bool post) {
   if (blocks > cap) blocks = cap;
   EventPair ep{};
   if (c->profiling) {
-    int rc = begin_timed(c, kClassFused, &ep);
+    int rc = begin_timed(c, kClassPeriod, &ep);
     if (rc) return rc;
   }
   k.fn<<<(unsigned)blocks, block, 0, c->stream>>>(pp);
@@ -467,8 +493,9 @@ int launch_period(la_ctx* c, uint32_t h, bool post) {
     LA_CUDA(c, cudaEventRecord(ep.b, c->stream));
     c->pending.push_back(ep);
   }
-  c->stats.launches_fused++;
-  c->stats.bytes_fused += pass_bytes(c, false, true, post, c->grad_kind);
+  const double bytes = pass_bytes(c, false, true, post, c->grad_kind);
+  c->stats.launches_fused++; c->stats.bytes_fused += bytes;
+  c->stats.launches_period++; c->stats.bytes_period += bytes;
   return LA_OK;
 }
 
@@ -490,6 +517,24 @@ int do_fill(la_ctx* c, const float* x0_dev) {
   la::la_fill<<<(unsigned)blocks, block, 0, c->stream>>>(c->X, c->B2, c->Bs, x0_dev, c->b0sq, c->stride, c->N, c->W);
   LA_CUDA(c, cudaGetLastError());
   c->stats.launches_other++;
+  return LA_OK;
+}
+
+// Algorithm 1 has ONE iterate that every worker holds; la_adagrad stores it in replica 0 only.
+// Before anything looks at replicas 1..W-1 individually again (another update rule, a per-worker
+// write), replica 0 is copied into them.
+int materialise_replicas(la_ctx* c) {
+  if (!c->shared_iterate) return LA_OK;
+  if (c->W > 1) {
+    const unsigned block = 256;
+    uint64_t blocks = (c->stride / 4 + block - 1) / block;
+    const uint64_t cap = (uint64_t)c->num_sms * 32;
+    if (blocks > cap) blocks = cap;
+    la::la_broadcast_replica0<<<(unsigned)blocks, block, 0, c->stream>>>(c->X, c->B2, c->stride, c->W);
+    LA_CUDA(c, cudaGetLastError());
+    c->stats.launches_other++;
+  }
+  c->shared_iterate = false;
   return LA_OK;
 }
 
@@ -609,6 +654,7 @@ int la_set_init(la_ctx* c, const float* x0_host, float b0sq) {
   }
   int rc = do_fill(c, x0_dev);
   if (rc) return rc;
+  c->shared_iterate = false;
   c->t = 0; c->tp = 0; c->nsync = 0;
   return LA_OK;
 }
@@ -675,6 +721,11 @@ int la_set_rule(la_ctx* c, int rule) {
   if (rule != LA_RULE_ADAALTER && rule != LA_RULE_LOCAL_SGD && rule != LA_RULE_ADAGRAD)
     return fail(c, LA_EINVAL, "unknown update rule %d", rule);
   if (c->tp != 0) return fail(c, LA_ESTATE, "the update rule can only change right after a synchronisation (t' = 0)");
+  if (c->rule == LA_RULE_ADAGRAD && rule != LA_RULE_ADAGRAD) {
+    DeviceGuard guard(c->device);
+    int rc = materialise_replicas(c);  // the other rules advance every replica on its own
+    if (rc) return rc;
+  }
   c->rule = rule;
   return LA_OK;
 }
@@ -713,7 +764,7 @@ int la_local_step(la_ctx* c) {
   int rc = launch_sweep(c, false, true, false, c->t + 1, c->tp + 1, c->grad_kind, nullptr);
   if (rc) return rc;
   c->t += 1;
-  if (c->rule == LA_RULE_ADAGRAD) c->nsync += 1;  // Algorithm 1 exchanges gradients every iteration
+  if (c->rule == LA_RULE_ADAGRAD) { c->nsync += 1; c->shared_iterate = true; }  // Algorithm 1 exchanges gradients every iteration
   else c->tp += 1;
   return LA_OK;
 }
@@ -727,7 +778,7 @@ int la_local_step_grads(la_ctx* c, const void* g_dev, int dtype) {
                         dtype == LA_F32 ? la::kGradExternalF32 : la::kGradExternalBF16, g_dev);
   if (rc) return rc;
   c->t += 1;
-  if (c->rule == LA_RULE_ADAGRAD) c->nsync += 1;
+  if (c->rule == LA_RULE_ADAGRAD) { c->nsync += 1; c->shared_iterate = true; }
   else c->tp += 1;
   return LA_OK;
 }
@@ -797,10 +848,14 @@ static int ensure_period_graph(la_ctx* c) {
   c->graph_delta.launches_local = c->stats.launches_local - st0.launches_local;
   c->graph_delta.launches_sync = c->stats.launches_sync - st0.launches_sync;
   c->graph_delta.launches_fused = c->stats.launches_fused - st0.launches_fused;
+  c->graph_delta.launches_step_sync = c->stats.launches_step_sync - st0.launches_step_sync;
+  c->graph_delta.launches_period = c->stats.launches_period - st0.launches_period;
   c->graph_delta.launches_other = 1;
   c->graph_delta.bytes_local = c->stats.bytes_local - st0.bytes_local;
   c->graph_delta.bytes_sync = c->stats.bytes_sync - st0.bytes_sync;
   c->graph_delta.bytes_fused = c->stats.bytes_fused - st0.bytes_fused;
+  c->graph_delta.bytes_step_sync = c->stats.bytes_step_sync - st0.bytes_step_sync;
+  c->graph_delta.bytes_period = c->stats.bytes_period - st0.bytes_period;
   c->stats = st0; c->t = t0; c->tp = tp0; c->nsync = ns0;
   if (rc != LA_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
   if (e != cudaSuccess || !graph) { cudaGetLastError(); return fail(c, LA_ECUDA, "stream capture failed: %s", cudaGetErrorString(e)); }
@@ -832,6 +887,10 @@ int la_run(la_ctx* c, uint64_t T) {
     c->stats.bytes_local += (double)reps * c->graph_delta.bytes_local;
     c->stats.bytes_sync += (double)reps * c->graph_delta.bytes_sync;
     c->stats.bytes_fused += (double)reps * c->graph_delta.bytes_fused;
+    c->stats.launches_step_sync += reps * c->graph_delta.launches_step_sync;
+    c->stats.launches_period += reps * c->graph_delta.launches_period;
+    c->stats.bytes_step_sync += (double)reps * c->graph_delta.bytes_step_sync;
+    c->stats.bytes_period += (double)reps * c->graph_delta.bytes_period;
     T -= reps * c->H;
   }
   return run_steps(c, T);
@@ -907,7 +966,7 @@ int la_read_range(la_ctx* c, uint32_t worker, uint64_t j0, uint64_t n, float* x_
   if (worker >= c->W) return fail(c, LA_EINVAL, "worker %u out of range (W=%u)", worker, c->W);
   if (j0 > c->N || n > c->N - j0) return fail(c, LA_EINVAL, "coordinate range out of bounds");
   DeviceGuard guard(c->device);
-  if (c->rule == LA_RULE_ADAGRAD) worker = 0;  // one shared iterate (Algorithm 1)
+  if (c->shared_iterate) worker = 0;  // Algorithm 1: every worker holds the one iterate, stored in replica 0
   const size_t bytes = n * sizeof(float);
   if (n) {
     if (x_host) LA_CUDA(c, cudaMemcpyAsync(x_host, c->X + (uint64_t)worker * c->stride + j0, bytes, cudaMemcpyDeviceToHost, c->stream));
@@ -927,6 +986,10 @@ int la_write_state(la_ctx* c, uint32_t worker, const float* x_host, const float*
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   if (worker >= c->W) return fail(c, LA_EINVAL, "worker %u out of range (W=%u)", worker, c->W);
   DeviceGuard guard(c->device);
+  if (x_host || b2_host) {
+    int rc = materialise_replicas(c);  // a per-worker write: the replicas become individual again
+    if (rc) return rc;
+  }
   const size_t bytes = c->N * sizeof(float);
   if (x_host) LA_CUDA(c, cudaMemcpyAsync(c->X + (uint64_t)worker * c->stride, x_host, bytes, cudaMemcpyHostToDevice, c->stream));
   if (b2_host) LA_CUDA(c, cudaMemcpyAsync(c->B2 + (uint64_t)worker * c->stride, b2_host, bytes, cudaMemcpyHostToDevice, c->stream));
@@ -981,6 +1044,10 @@ int la_comm_create(la_ctx* c, uint32_t rank, uint32_t world) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   if (world == 0 || world > la::kMaxRanks || rank >= world) return fail(c, LA_EINVAL, "need rank < world <= %d", la::kMaxRanks);
   if (c->rule != LA_RULE_ADAALTER) return fail(c, LA_ESTATE, "sharding by worker is implemented for Local AdaAlter only");
+  // "tree over the local replicas, then tree over the ranks" is the adjacent-pair tree over all
+  // workers only when every rank contributes a full power-of-two block of leaves
+  if (world > 1 && (c->W & (c->W - 1)) != 0)
+    return fail(c, LA_EINVAL, "with more than one rank the local worker count must be a power of two (W=%u)", c->W);
   DeviceGuard guard(c->device);
   if (!c->S) {
     cudaError_t e = cudaMalloc((void**)&c->S, 2 * c->stride * sizeof(float));
@@ -1181,7 +1248,7 @@ int la_diagnostics(la_ctx* c, double* objective, double* replica_spread) {
   }
   LA_CUDA(c, cudaMemsetAsync(c->diag, 0, 2 * sizeof(double), c->stream));
   const bool quad = c->grad_kind == la::kGradQuadratic;
-  const uint32_t W = c->rule == LA_RULE_ADAGRAD ? 1u : c->W;  // AdaGrad keeps one shared iterate
+  const uint32_t W = c->shared_iterate ? 1u : c->W;  // after AdaGrad steps all workers hold replica 0's iterate
   uint64_t blocks = (c->N + la::kBlockThreads - 1) / la::kBlockThreads;
   const uint64_t cap = (uint64_t)c->num_sms * 16;
   if (blocks > cap) blocks = cap;

@@ -27,7 +27,6 @@ static __device__ __align__(256) float g_static_sums[2 * kMaxCoords];
 std::mutex g_mutex;
 float* g_scratch_addr[kMaxDevices] = {};  // device address of g_static_sums, per device ordinal
 
-template <int V>
 __global__ void __launch_bounds__(LA_BLOCK) la_scale_sums(const float* __restrict__ sums, uint64_t sums_stride,
                                                           float* __restrict__ x_mean, float* __restrict__ b2_mean,
                                                           uint64_t n, uint32_t W) {
@@ -55,9 +54,11 @@ extern "C" int la_replica_means_static(const float* x_dev, const float* b2_dev, 
     // once per device, with that device current: resolve the array's device address
     std::lock_guard<std::mutex> lock(g_mutex);
     if (!g_scratch_addr[dev]) {
+      // With lazy module loading (CUDA's default) this is also the moment the driver reserves the
+      // array's 8 MiB on this device.  On failure nothing is cached, so a later call tries again.
       void* p = nullptr;
       if (cudaGetSymbolAddress(&p, g_static_sums) != cudaSuccess || !p) {
-        cudaGetLastError();
+        cudaGetLastError();  // clear the error so that it does not surface in the caller's next CUDA call
         return LA_ECUDA;
       }
       g_scratch_addr[dev] = static_cast<float*>(p);
@@ -80,7 +81,7 @@ extern "C" int la_replica_means_static(const float* x_dev, const float* b2_dev, 
   if (cudaGetLastError() != cudaSuccess) return LA_ECUDA;
   uint64_t blocks2 = (n + block - 1) / block;
   if (blocks2 > (1u << 20)) blocks2 = 1u << 20;
-  la_scale_sums<1><<<(unsigned)blocks2, block, 0, st>>>(scratch, stride, x_mean_dev, b2_mean_dev, n, W);
+  la_scale_sums<<<(unsigned)blocks2, block, 0, st>>>(scratch, stride, x_mean_dev, b2_mean_dev, n, W);
   if (cudaGetLastError() != cudaSuccess) return LA_ECUDA;
   return LA_OK;
 }

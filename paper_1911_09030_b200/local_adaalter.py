@@ -36,7 +36,11 @@ class la_stats(C.Structure):
     _fields_ = [("launches_local", C.c_uint64), ("launches_sync", C.c_uint64),
                 ("launches_fused", C.c_uint64), ("launches_other", C.c_uint64),
                 ("ms_local", C.c_double), ("ms_sync", C.c_double), ("ms_fused", C.c_double),
-                ("bytes_local", C.c_double), ("bytes_sync", C.c_double), ("bytes_fused", C.c_double)]
+                ("bytes_local", C.c_double), ("bytes_sync", C.c_double), ("bytes_fused", C.c_double),
+                ("launches_step_sync", C.c_uint64), ("launches_sync_step", C.c_uint64),
+                ("launches_period", C.c_uint64),
+                ("ms_step_sync", C.c_double), ("ms_sync_step", C.c_double), ("ms_period", C.c_double),
+                ("bytes_step_sync", C.c_double), ("bytes_sync_step", C.c_double), ("bytes_period", C.c_double)]
 
 
 _lib = None

@@ -9,7 +9,8 @@ library; this module only orders the phases of a synchronisation and moves handl
       "peer":      stream sync + barrier, `combine` (each rank reduces its coordinate slice over
                    all ranks' buffers with peer loads and writes the total back to all), stream
                    sync + barrier
-      "allreduce": one all-reduce(SUM) of the exchange buffer by torch.distributed (NCCL)
+      "allreduce": stream sync, one all-reduce(SUM) of the exchange buffer by torch.distributed
+                   (NCCL), wait for it
     import  (total / W_total -> every local replica, stale accumulator; t' = 0)
 
 The engine is anything with the methods used below; the CUDA engine is `CudaEngine`.
@@ -51,7 +52,14 @@ class WorkerShardedJob:
         else:
             buf = e.buffer_tensor()
             if self.dist is not None and self.dist.is_initialized() and self.dist.get_world_size(self.group) > 1:
+                # The export kernel ran on the context's stream, the collective runs on the process
+                # group's: finish the first before the second reads the buffer, and finish the second
+                # before the import kernel (context stream again) reads the totals.
+                e.stream_sync()
                 self.dist.all_reduce(buf, op=self.dist.ReduceOp.SUM, group=self.group)
+                done = getattr(e, "collective_done", None)
+                if done is not None:
+                    done()
 
     def run(self, T: int):
         """T iterations of Algorithm 3: local step; if t' == H: synchronise."""
@@ -122,6 +130,11 @@ class CudaEngine:
 
     def stream_sync(self):
         self.ctx.stream_sync()
+
+    def collective_done(self):
+        """Block until the collective torch enqueued on its current stream has finished."""
+        import torch
+        torch.cuda.current_stream().synchronize()
 
     def buffer_tensor(self):
         if self._tensor is None:

@@ -67,13 +67,22 @@ def _chunk(seed: int, which: int, chunk: int, draw) -> np.ndarray:
 
 def _range_of(seed: int, which: int, j0: int, n: int, draw) -> np.ndarray:
     out = np.empty(n, np.float32)
-    j = j0
-    while j < j0 + n:
-        ch = j // CHUNK
-        lo = j - ch * CHUNK
-        hi = min(CHUNK, j0 + n - ch * CHUNK)
-        out[j - j0: j - j0 + (hi - lo)] = _chunk(seed, which, ch, draw)[lo:hi]
-        j += hi - lo
+    first, last = j0 // CHUNK, (j0 + n - 1) // CHUNK if n else j0 // CHUNK - 1
+
+    def fill(ch: int) -> None:
+        lo = max(j0, ch * CHUNK)
+        hi = min(j0 + n, (ch + 1) * CHUNK)
+        out[lo - j0: hi - j0] = _chunk(seed, which, ch, draw)[lo - ch * CHUNK: hi - ch * CHUNK]
+
+    chunks = range(first, last + 1)
+    if len(chunks) > 8:      # chunks are independent streams: draw them on several host threads
+        import os
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as ex:
+            list(ex.map(fill, chunks))
+    else:
+        for ch in chunks:
+            fill(ch)
     return out
 
 

@@ -44,7 +44,7 @@ def test_struct_layout_matches_header():
     from paper_1911_09030_b200 import local_adaalter as la
     # natural alignment of the C struct: u32, ptr, u64, u32 x2, f32 x3, ptr, u64, ptr, i32
     assert C.sizeof(la.la_config) == 80
-    assert C.sizeof(la.la_stats) == 4 * 8 + 6 * 8
+    assert C.sizeof(la.la_stats) == 4 * 8 + 6 * 8 + 3 * 8 + 6 * 8
 
 
 @pytest.mark.parametrize("kw,frag", [

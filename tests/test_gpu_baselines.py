@@ -50,6 +50,46 @@ def test_adagrad_matches_oracle(W, grad):
         g.sync()
 
 
+@pytest.mark.parametrize("W", [3, 8])
+@pytest.mark.parametrize("next_rule", [la.LA_RULE_ADAALTER, la.LA_RULE_LOCAL_SGD])
+def test_leaving_adagrad_continues_from_the_common_iterate(W, next_rule):
+    """Algorithm 1 keeps one iterate that every worker holds.  When another rule takes over, every
+    replica must start from it (and from the common accumulator), as in the oracle."""
+    n, H = 3001, 4
+    arr = _arrays(n, 40 + W)
+    g, o = make_pair(n, W, 0.2, 0.5, H, "quadratic", seed=8, arrays=arr, sigma=0.7)
+    g.run(H); o.run(H)                                    # replicas have a history of their own first
+    g.set_rule(la.LA_RULE_ADAGRAD); o.set_rule(2)
+    g.run(3); o.run(3)
+    compare(g, o, W, 1e-5)
+    g.set_rule(next_rule); o.set_rule(next_rule)
+    compare(g, o, W, 1e-5)                                # every worker reads the common iterate
+    g.run(H + 1); o.run(H + 1)
+    compare(g, o, W, 1e-5)
+    g.run(H - 1); o.run(H - 1)
+    g.set_rule(la.LA_RULE_ADAGRAD); o.set_rule(2)         # and back again
+    g.run(2); o.run(2)
+    compare(g, o, W, 1e-5)
+    g.close()
+
+
+def test_state_written_per_worker_under_adagrad_is_kept():
+    """A per-worker write after AdaGrad steps makes the replicas individual again."""
+    n, W = 515, 4
+    arr = _arrays(n, 3)
+    g, o = make_pair(n, W, 0.2, 0.5, 2, "noise_scaled", seed=4, arrays=arr)
+    g.set_rule(la.LA_RULE_ADAGRAD); o.set_rule(2)
+    g.run(2); o.run(2)
+    x = np.linspace(-1, 1, n).astype(np.float32)
+    b = np.full(n, 2.5, np.float32)
+    g.write_state(2, x, b, None); o.write(2, x, b, None)
+    compare(g, o, W, 0.0)
+    g.set_rule(la.LA_RULE_ADAALTER); o.set_rule(0)
+    g.run(3); o.run(3)
+    compare(g, o, W, 1e-5)
+    g.close()
+
+
 def test_rule_changes_only_at_a_period_boundary():
     g = la.LocalAdaAlter([64], 2, 0.1, 1.0, 4)
     g.set_grad_noise(1)

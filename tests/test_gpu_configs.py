@@ -122,32 +122,73 @@ def test_beyond_32_bit_indexing():
     g.close()
 
 
-def test_config2_four_million_coordinates_full_run():
-    """Configuration 2, full W and T, on 2^22 coordinates (64 blocks of 2^16 spread evenly over the
-    vector), the oracle running one block per host thread."""
+def _deep_ranges(wl, nblocks=64, block=1 << 16, ends=4096, around=8):
+    """At least 2^22 coordinates of the full-size vector: `nblocks` blocks spread evenly (so that
+    every part of the grid is hit), both ends, and a window around every tensor boundary."""
+    N = wl.N
+    want = [(0, min(ends, N)), (max(0, (N - ends) // 4 * 4), N)]
+    step = N // nblocks
+    for k in range(nblocks):
+        lo = (k * step) // 4 * 4
+        want.append((lo, min(N, lo + block)))
+    off = 0
+    for sz in wl.sizes[:-1]:
+        off += sz
+        lo = max(0, (off - around) // 4 * 4)
+        want.append((lo, min(N, lo + 2 * around + 4)))
+    want.sort()
+    merged = []
+    for lo, hi in want:
+        if merged and lo <= merged[-1][1]:
+            merged[-1] = (merged[-1][0], max(merged[-1][1], hi))
+        else:
+            merged.append((lo, hi))
+    return merged
+
+
+DEEP_CASES = [("c2", None, (1, 3)), ("c3", None, (1, 3)), ("c5", None, (1, 3)),
+              ("c4", 1, (2,)), ("c4", 4, (0,)), ("c4", 16, (1, 3)), ("c4", 64, (2,))]
+
+
+@pytest.mark.parametrize("name,H,fusions", DEEP_CASES, ids=[f"{n}-H{h}-f{''.join(map(str, f))}" for n, h, f in DEEP_CASES])
+def test_full_size_run_on_four_million_coordinates(name, H, fusions):
+    """Each configuration at full size, full W and T, in the launch configuration the benchmark
+    times; the oracle re-computes >= 2^22 coordinates (blocks spread over the whole vector, both
+    ends, every tensor boundary), one block per host thread; every x, B^2 and stale B^2 of every
+    worker must agree bit for bit.  One oracle pass serves all fusion modes of a case."""
     import os
-    from concurrent.futures import ThreadPoolExecutor
-    wl = workloads.config("c2")
-    arr = wl.arrays()
-    g = _make_gpu(wl, arr, wl.H, la.LA_FUSE_STEP_SYNC)
-    g.run(wl.T)
-    blocks = [(k * (wl.N // 64), k * (wl.N // 64) + (1 << 16)) for k in range(64)]
     import threading
+    from concurrent.futures import ThreadPoolExecutor
+    wl = workloads.config(name)
+    H = wl.H if H is None else H
+    arr = wl.arrays()
+    gpus = []
+    for fusion in fusions:
+        g = _make_gpu(wl, arr, H, fusion)
+        g.run(wl.T)
+        assert g.get_counters() == (wl.T, wl.T % H, wl.T // H)
+        gpus.append(g)
+    ranges = _deep_ranges(wl)
+    assert sum(hi - lo for lo, hi in ranges) >= 1 << 22
     ctx_lock = threading.Lock()                      # a context serves one caller thread at a time
 
     def check(rng):
         lo, hi = rng
-        o = _make_oracle(wl, arr, wl.H, lo, hi)
+        o = _make_oracle(wl, arr, H, lo, hi)
         o.run(wl.T)
         bad = 0
         for i in range(wl.W):
-            with ctx_lock:
-                got = g.read_range(i, lo, hi - lo)
-            for a, b in zip(got, o.read(i)):
-                bad += int(np.count_nonzero(a.view(np.uint32) != b.view(np.uint32)))
+            ref = o.read(i)
+            for g in gpus:
+                with ctx_lock:
+                    got = g.read_range(i, lo, hi - lo)
+                for a, b in zip(got, ref):
+                    bad += int(np.count_nonzero(a.view(np.uint32) != b.view(np.uint32)))
+        o.close()
         return bad
 
-    with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as ex:
-        mismatches = sum(ex.map(check, blocks))
+    with ThreadPoolExecutor(max_workers=min(32, os.cpu_count() or 1)) as ex:
+        mismatches = sum(ex.map(check, ranges))
     assert mismatches == 0
-    g.close()
+    for g in gpus:
+        g.close()

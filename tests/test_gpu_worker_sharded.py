@@ -111,6 +111,12 @@ def test_misuse_is_reported():
         g.comm_create(3, 2)
     with pytest.raises(la.LocalAdaAlterError):
         g.set_worker_range(7, 8)
+    # three local workers on each of two ranks would not reproduce the adjacent-pair tree over six
+    g3 = la.LocalAdaAlter([64], 3, 0.1, 1.0, 2)
+    with pytest.raises(la.LocalAdaAlterError) as e:
+        g3.comm_create(0, 2)
+    assert e.value.code == la.LA_EINVAL and "power of two" in str(e.value)
+    g3.comm_create(0, 1)                     # a single rank may hold any number of workers
 
 
 TWO_PROCESS = r'''
