@@ -250,6 +250,14 @@ int la_comm_import(la_ctx* ctx);
 int la_comm_step_export(la_ctx* ctx);
 int la_comm_step_grads_export(la_ctx* ctx, const void* g_dev, int dtype);
 int la_comm_import_step(la_ctx* ctx);
+/* Verification aid for the synthetic gradient source (not part of the paper's method): the two
+ * building blocks of the normal draw, exactly as the sweep kernels evaluate them, over their whole
+ * 24-bit domains, so that they can be compared element by element with another implementation:
+ *   radius_dev[k-1] = sqrt(-2 ln(k 2^-24)), k = 1..2^24
+ *   cos_dev[q], sin_dev[q] = cos, sin(2 pi q 2^-24), q = 0..2^24-1
+ * Each pointer is device memory for 2^24 floats, or NULL to skip that table.  Enqueued on
+ * `stream` (a cudaStream_t, NULL = default) of the current device; needs no context. */
+int la_noise_tables(float* radius_dev, float* cos_dev, float* sin_dev, void* stream);
 /* Block until the context's stream is idle. */
 int la_stream_sync(la_ctx* ctx);
 

@@ -520,6 +520,21 @@ void ora_scan_neg2ln(double* out) {
   }
   out[0] = maxabs; out[1] = maxrel; out[2] = minL; out[3] = (double)neg2ln_u24(1u << 24);
 }
+// Whole-domain tables of the two building blocks of the noise recipe, for element-by-element
+// comparison with another implementation: L[k-1] = neg2ln_u24(k), k = 1..2^24, and
+// (c[q], s[q]) = cossin_u24(q), q = 0..2^24-1.  Any pointer may be null.
+void ora_table_neg2ln(float* L) {
+  if (!L) return;
+  for (uint32_t k = 1; k <= (1u << 24); ++k) L[k - 1] = neg2ln_u24(k);
+}
+void ora_table_cossin(float* c, float* s) {
+  for (uint32_t q = 0; q < (1u << 24); ++q) {
+    float cc, ss;
+    cossin_u24(q, &cc, &ss);
+    if (c) c[q] = cc;
+    if (s) s[q] = ss;
+  }
+}
 // out[0] = max abs error of cos, out[1] = of sin, out[2] = max |c^2+s^2-1|.
 void ora_scan_cossin(double* out) {
   double ec = 0, es = 0, en = 0;

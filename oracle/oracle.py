@@ -85,6 +85,8 @@ def lib() -> C.CDLL:
             L.ora_uniform_bits.argtypes = [u64, u64, u32, u64, vp, vp]
             L.ora_scan_neg2ln.argtypes = [vp]
             L.ora_scan_cossin.argtypes = [vp]
+            L.ora_table_neg2ln.argtypes = [vp]
+            L.ora_table_cossin.argtypes = [vp, vp]
             _lib = L
     return _lib
 
@@ -241,6 +243,20 @@ def scan_neg2ln():
     out = np.zeros(4, np.float64)
     lib().ora_scan_neg2ln(_ptr(out))
     return dict(max_abs=out[0], max_rel=out[1], min_L=out[2], L_at_one=out[3])
+
+
+def table_neg2ln():
+    """L[k-1] = -2 ln(k 2^-24) by the recipe, for every k in 1..2^24."""
+    out = np.empty(1 << 24, np.float32)
+    lib().ora_table_neg2ln(_ptr(out))
+    return out
+
+
+def table_cossin():
+    """(cos, sin)(2 pi q 2^-24) by the recipe, for every q in 0..2^24-1."""
+    c, s = np.empty(1 << 24, np.float32), np.empty(1 << 24, np.float32)
+    lib().ora_table_cossin(_ptr(c), _ptr(s))
+    return c, s
 
 
 def scan_cossin():

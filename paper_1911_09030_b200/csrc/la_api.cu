@@ -154,6 +154,22 @@ __global__ void la_broadcast_replica0(float* X, float* B2, uint64_t stride, uint
   }
 }
 
+// The two building blocks of the noise source over their whole 24-bit domains, as the sweep
+// kernels evaluate them: radius[k-1] = sqrt(-2 ln(k 2^-24)), k = 1..2^24; (cos, sin)(2 pi q 2^-24),
+// q = 0..2^24-1.
+__global__ void la_noise_tables_kernel(float* radius, float* cs, float* sn) {
+  const uint32_t nthreads = gridDim.x * blockDim.x;
+  for (uint32_t q = blockIdx.x * blockDim.x + threadIdx.x; q < (1u << 24); q += nthreads) {
+    if (radius) radius[q] = radius_from_u24(q + 1u);
+    if (cs || sn) {
+      float c, s;
+      cossin_from_top24(q << 8, c, s);
+      if (cs) cs[q] = c;
+      if (sn) sn[q] = s;
+    }
+  }
+}
+
 // Device-resident step counter used by captured graphs (see la_set_graph).
 __global__ void la_counter_set(uint64_t* ctr, uint64_t v) { *ctr = v; }
 __global__ void la_counter_add(uint64_t* ctr, uint64_t v) { *ctr += v; }
@@ -474,13 +490,13 @@ int launch_period(la_ctx* c, uint32_t h, bool post) {
   p.worker_base = c->worker_base;
   p.eta = c->eta; p.eps = c->eps; p.sigma = c->sigma;
   pp.h = h;
-  const unsigned block = la::kBlockThreads;
+  const unsigned block = (unsigned)k.block;
   const uint64_t ngroups = (c->N + (uint64_t)k.vec - 1) / (uint64_t)k.vec;
   uint64_t blocks = (ngroups + block - 1) / block;
   // issue-bound kernel: at the full configuration sizes 384..768 blocks per SM in the grid measured
   // best (few coordinate groups per thread); smaller grids lose up to 20 %
-  const int bps = c->blocks_per_sm > 0 ? c->blocks_per_sm : 768;
-  const uint64_t cap = (uint64_t)c->num_sms * (uint64_t)bps;
+  const int bps = c->blocks_per_sm > 0 ? c->blocks_per_sm : 768;  // counted in 256-thread units
+  const uint64_t cap = (uint64_t)c->num_sms * (uint64_t)bps * 256u / block;
   if (blocks > cap) blocks = cap;
   EventPair ep{};
   if (c->profiling) {
@@ -1261,6 +1277,13 @@ int la_diagnostics(la_ctx* c, double* objective, double* replica_spread) {
   LA_CUDA(c, cudaStreamSynchronize(c->stream));
   if (objective) *objective = quad ? host[0] : NAN;
   if (replica_spread) *replica_spread = host[1];
+  return LA_OK;
+}
+
+int la_noise_tables(float* radius_dev, float* cos_dev, float* sin_dev, void* stream) {
+  if (!radius_dev && !cos_dev && !sin_dev) return LA_OK;
+  la::la_noise_tables_kernel<<<148 * 8, 256, 0, (cudaStream_t)stream>>>(radius_dev, cos_dev, sin_dev);
+  if (cudaGetLastError() != cudaSuccess) return fail(nullptr, LA_ECUDA, "launch of the table kernel failed");
   return LA_OK;
 }
 

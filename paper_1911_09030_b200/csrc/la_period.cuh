@@ -14,6 +14,12 @@
 #ifndef LA_PERIOD_UNROLL
 #define LA_PERIOD_UNROLL 2
 #endif
+#ifndef LA_PERIOD_BLOCK
+#define LA_PERIOD_BLOCK LA_BLOCK
+#endif
+#ifndef LA_PERIOD_CH
+#define LA_PERIOD_CH 8  // replicas whose gradient chains are interleaved
+#endif
 
 namespace la {
 
@@ -26,10 +32,10 @@ struct PeriodParams {
 };
 
 template <int W_, int V, int GM, bool BF16, bool POST, int MINB>
-__global__ void __launch_bounds__(LA_BLOCK, MINB) la_period(const PeriodParams pp) {
+__global__ void __launch_bounds__(LA_PERIOD_BLOCK, MINB) la_period(const PeriodParams pp) {
   const SweepParams& p = pp.base;
   constexpr bool kNeedsNoise = (GM == kGradNoise || GM == kGradNoiseScaled || GM == kGradQuadratic);
-  constexpr int CH = (W_ > 0) ? (W_ < LA_CH ? W_ : LA_CH) : 4;
+  constexpr int CH = (W_ > 0) ? (W_ < LA_PERIOD_CH ? W_ : LA_PERIOD_CH) : 4;
   constexpr int kOuterUnroll = (W_ > 0) ? kMaxWorkers : 1;
   const uint32_t W = (W_ > 0) ? (uint32_t)W_ : p.W;
   const uint32_t h = pp.h;
@@ -37,7 +43,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_period(const PeriodParams p
   // stream keys of every (step, worker) of this pass, and the per-step scalars
   __shared__ uint64_t keys[kPeriodMax][kMaxWorkers];
   __shared__ float eta_s[kPeriodMax], q_s[kPeriodMax];
-  __shared__ Vec<V> r_s[kPeriodMax][LA_BLOCK];
+  __shared__ Vec<V> r_s[kPeriodMax][LA_PERIOD_BLOCK];
   if (kNeedsNoise) {
     for (uint32_t k = threadIdx.x; k < h * W; k += blockDim.x) {
       const uint32_t s = k / W, i = k - s * W;
@@ -59,25 +65,21 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_period(const PeriodParams p
 
   const uint64_t ngroups = (p.n + (uint64_t)(V - 1)) / (uint64_t)V;
   const uint64_t nthreads = (uint64_t)gridDim.x * blockDim.x;
-  uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (grp >= ngroups) return;
   const uint64_t x_base = reinterpret_cast<uint64_t>(p.X);
   const uint64_t b_delta = reinterpret_cast<uint64_t>(p.B2) - x_base;
   const uint64_t stride_bytes = p.stride * sizeof(float);
 
-  ReplicaChunk<V, CH> nxt;
-  CoordInputs<V> in_next;
-  load_coord<GM, true, true, V>(in_next, p, grp * V);
-  uint64_t ld_addr = x_base + grp * (V * sizeof(float));
-  load_chunk<V, CH>(nxt, ld_addr, b_delta, stride_bytes, W, 0u);
-
-  for (;;) {
+  // The kernel is bound by instruction issue, not by HBM (a sixth of the bandwidth is in use), so
+  // unlike la_sweep it does not prefetch the next chunk while one is processed: the registers that
+  // would hold loads in flight are worth more as room for interleaving the gradient chains, and
+  // the other resident blocks cover the load latency.
+  for (uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < ngroups; grp += nthreads) {
     const uint64_t off = grp * V;
-    const uint64_t next_grp = grp + nthreads;
-    const bool has_next = next_grp < ngroups;
-    const CoordInputs<V> in = in_next;
+    CoordInputs<V> in;
+    load_coord<GM, true, true, V>(in, p, off);
     const uint64_t ctr0 = kGoldenGamma * (((p.j_base + off) >> 1) + 1u);
-    uint64_t st_addr = x_base + off * sizeof(float);
+    uint64_t ld_addr = x_base + off * sizeof(float);
+    uint64_t st_addr = ld_addr;
 
     // step sizes of the h steps: the stale accumulator is fixed, only t' eps^2 ramps.  They live
     // in this thread's own shared-memory column so that the loop over steps can stay rolled: with
@@ -88,26 +90,25 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_period(const PeriodParams p
 
 #pragma unroll kOuterUnroll
     for (uint32_t i0 = 0; i0 < W; i0 += CH) {
-      ReplicaChunk<V, CH> cur = nxt;
-      if (i0 + CH < W) {
-        load_chunk<V, CH>(nxt, ld_addr, b_delta, stride_bytes, W, i0 + CH);
-      } else if (has_next) {
-        load_coord<GM, true, true, V>(in_next, p, next_grp * V);
-        ld_addr = x_base + next_grp * (V * sizeof(float));
-        load_chunk<V, CH>(nxt, ld_addr, b_delta, stride_bytes, W, 0u);
+      ReplicaChunk<V, CH> cur;
+      load_chunk<V, CH>(cur, ld_addr, b_delta, stride_bytes, W, i0);
+      // steps outside, the chunk's replicas inside: CH independent gradient chains per iteration
+#pragma unroll kPeriodUnroll
+      for (uint32_t s = 0; s < h; ++s) {
+        const Vec<V> r = r_s[s][threadIdx.x];
+#pragma unroll
+        for (int k = 0; k < CH; ++k)
+          if (i0 + k < W) {
+            const uint32_t i = i0 + k;
+            const Vec<V> g = gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[s][i] : 0ull, ctr0, i, off);
+            apply<V>(r, g, cur.x[k], cur.b[k]);
+          }
       }
-      asm volatile("" ::: "memory");
 #pragma unroll
       for (int k = 0; k < CH; ++k)
         if (i0 + k < W) {
-          const uint32_t i = i0 + k;
-#pragma unroll kPeriodUnroll
-          for (uint32_t s = 0; s < h; ++s) {
-            const Vec<V> g = gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[s][i] : 0ull, ctr0, i, off);
-            apply<V>(r_s[s][threadIdx.x], g, cur.x[k], cur.b[k]);
-          }
           if (POST) {
-            tree.push_in_chunk(i, k, i0 + CH <= W, cur.x[k], cur.b[k]);
+            tree.push_in_chunk(i0 + k, k, i0 + CH <= W, cur.x[k], cur.b[k]);
           } else {
             store_replica<V>(st_addr, b_delta, stride_bytes, cur.x[k], cur.b[k]);
           }
@@ -121,8 +122,6 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_period(const PeriodParams p
 #pragma unroll kOuterUnroll
       for (uint32_t i = 0; i < W; ++i) store_replica<V>(st_addr, b_delta, stride_bytes, xm, bm);
     }
-    if (!has_next) break;
-    grp = next_grp;
   }
 }
 
@@ -130,6 +129,7 @@ using PeriodFn = void (*)(const PeriodParams);
 struct PeriodKernel {
   PeriodFn fn;
   int vec;
+  int block;  // threads per block the kernel was compiled for
 };
 PeriodKernel lookup_period(int W, int gm, bool bf16, bool post);
 

@@ -407,7 +407,10 @@ __device__ __forceinline__ Vec<V> gradient(const SweepParams& p, const CoordInpu
       } else {  // quadratic
         g.v[k] = __fmaf_rn(in.a.v[k], __fsub_rn(xv.v[k], in.c.v[k]), __fmul_rn(p.sigma, xi.v[k]));
       }
-      if (BF16) g.v[k] = round_through_bf16(g.v[k]);
+    }
+    if (BF16) {
+#pragma unroll
+      for (int k = 0; k < V; k += 2) round_pair_through_bf16(g.v[k], g.v[k + 1]);
     }
   }
   return g;

@@ -98,6 +98,7 @@ def lib() -> C.CDLL:
             "la_comm_step_grads_export": [vp, vp, i32],
             "la_comm_import_step": [vp],
             "la_stream_sync": [vp],
+            "la_noise_tables": [vp, vp, vp, vp],
             "la_replica_means_static": [vp, vp, u32, u64, u64, vp, vp, vp],
         }
         for name, args in sig.items():
@@ -118,6 +119,12 @@ def replica_means_static(x_ptr, b2_ptr, W, n, stride, x_mean_ptr, b2_mean_ptr, s
     return lib().la_replica_means_static(C.c_void_p(int(x_ptr)), C.c_void_p(int(b2_ptr)), int(W), int(n), int(stride),
                                          C.c_void_p(int(x_mean_ptr)), C.c_void_p(int(b2_mean_ptr)),
                                          C.c_void_p(int(stream)) if stream else None)
+
+
+def noise_tables(radius_ptr=None, cos_ptr=None, sin_ptr=None, stream=None) -> int:
+    """`la_noise_tables`: fill device buffers of 2^24 floats each (raw addresses, None to skip)."""
+    vp = lambda p: C.c_void_p(int(p)) if p else None
+    return lib().la_noise_tables(vp(radius_ptr), vp(cos_ptr), vp(sin_ptr), vp(stream))
 
 
 class LocalAdaAlterError(RuntimeError):

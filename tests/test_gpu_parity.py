@@ -561,3 +561,24 @@ def test_run_time_worker_counts_over_many_blocks(W):
         g.run(T); o.run(T)
         compare(g, o, W, TOL_RUN)
         g.close()
+
+
+def test_noise_building_blocks_over_their_whole_domain():
+    """Every one of the 2^24 radii and 2^24 (cos, sin) pairs the kernels can produce, against the
+    oracle's recipe, bit for bit.  The radius is sqrt(L) with L from the oracle's table and the
+    correctly rounded fp32 square root (numpy's), which is what the oracle's noise draw applies."""
+    import torch
+    from oracle import oracle as O
+    r = torch.empty(1 << 24, dtype=torch.float32, device="cuda")
+    c = torch.empty_like(r)
+    s = torch.empty_like(r)
+    assert la.noise_tables(r.data_ptr(), c.data_ptr(), s.data_ptr()) == la.LA_OK
+    torch.cuda.synchronize()
+    L = O.table_neg2ln()
+    assert L.min() >= 0.0 and L[-1] == 0.0
+    want_r = np.sqrt(L, dtype=np.float32)
+    assert np.array_equal(r.cpu().numpy().view(np.uint32), want_r.view(np.uint32))
+    oc, os_ = O.table_cossin()
+    assert np.array_equal(c.cpu().numpy().view(np.uint32), oc.view(np.uint32))
+    assert np.array_equal(s.cpu().numpy().view(np.uint32), os_.view(np.uint32))
+    assert la.noise_tables(None, None, None) == la.LA_OK

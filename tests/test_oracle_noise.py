@@ -164,3 +164,16 @@ def test_gradient_modes_against_their_definitions():
                 # accumulated g^2 is the square of a bf16-representable number
                 back = torch.from_numpy(gg.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
                 np.testing.assert_allclose(gg, back, rtol=1e-5, atol=1e-4)
+
+
+def test_whole_domain_tables_are_the_scalar_recipes():
+    """The table accessors only loop over the pinned scalar functions."""
+    L = O.table_neg2ln()
+    c, s = O.table_cossin()
+    rng = np.random.default_rng(5)
+    for k in [1, 2, 3, (1 << 24) - 1, 1 << 24] + [int(v) for v in rng.integers(1, 1 << 24, 200)]:
+        assert L[k - 1] == np.float32(O.neg2ln_u24(k))
+    for q in [0, 1, (1 << 21) - 1, 1 << 21, (1 << 24) - 1] + [int(v) for v in rng.integers(0, 1 << 24, 200)]:
+        cc, ss = O.cossin_u24(q)
+        assert c[q] == np.float32(cc) and s[q] == np.float32(ss)
+    assert L[-1] == 0.0 and np.all(L[:-1] > 0) and np.all(np.diff(L.astype(np.float64)) <= 0)
