@@ -18,27 +18,27 @@
 
 namespace la {
 
-SweepKernel lookup_sweep_w0(int, int, bool, bool, bool, bool);
-SweepKernel lookup_sweep_w1(int, int, bool, bool, bool, bool);
-SweepKernel lookup_sweep_w2(int, int, bool, bool, bool, bool);
-SweepKernel lookup_sweep_w4(int, int, bool, bool, bool, bool);
-SweepKernel lookup_sweep_w8(int, int, bool, bool, bool, bool);
-SweepKernel lookup_sweep_w16(int, int, bool, bool, bool, bool);
-SweepKernel lookup_sweep_w3(int, int, bool, bool, bool, bool);
-SweepKernel lookup_sweep_w6(int, int, bool, bool, bool, bool);
-SweepKernel lookup_sweep_w12(int, int, bool, bool, bool, bool);
+SweepKernel lookup_sweep_w0(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w1(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w2(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w4(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w8(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w16(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w3(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w6(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w12(int, int, bool, bool, bool, bool, int);
 
-SweepKernel lookup_sweep(int W, int rule, int gm, bool bf16, bool pre, bool step, bool post) {
+SweepKernel lookup_sweep(int W, int rule, int gm, bool bf16, bool pre, bool step, bool post, int xch) {
   switch (W) {
-    case 1: return lookup_sweep_w1(rule, gm, bf16, pre, step, post);
-    case 2: return lookup_sweep_w2(rule, gm, bf16, pre, step, post);
-    case 4: return lookup_sweep_w4(rule, gm, bf16, pre, step, post);
-    case 8: return lookup_sweep_w8(rule, gm, bf16, pre, step, post);
-    case 16: return lookup_sweep_w16(rule, gm, bf16, pre, step, post);
-    case 3: return lookup_sweep_w3(rule, gm, bf16, pre, step, post);
-    case 6: return lookup_sweep_w6(rule, gm, bf16, pre, step, post);
-    case 12: return lookup_sweep_w12(rule, gm, bf16, pre, step, post);
-    default: return lookup_sweep_w0(rule, gm, bf16, pre, step, post);
+    case 1: return lookup_sweep_w1(rule, gm, bf16, pre, step, post, xch);
+    case 2: return lookup_sweep_w2(rule, gm, bf16, pre, step, post, xch);
+    case 4: return lookup_sweep_w4(rule, gm, bf16, pre, step, post, xch);
+    case 8: return lookup_sweep_w8(rule, gm, bf16, pre, step, post, xch);
+    case 16: return lookup_sweep_w16(rule, gm, bf16, pre, step, post, xch);
+    case 3: return lookup_sweep_w3(rule, gm, bf16, pre, step, post, xch);
+    case 6: return lookup_sweep_w6(rule, gm, bf16, pre, step, post, xch);
+    case 12: return lookup_sweep_w12(rule, gm, bf16, pre, step, post, xch);
+    default: return lookup_sweep_w0(rule, gm, bf16, pre, step, post, xch);
   }
 }
 
@@ -66,64 +66,7 @@ PeriodKernel lookup_period(int W, int gm, bool bf16, bool post) {
   }
 }
 
-#define LA_DECL_XCH(w)                                   \
-  StepExportFn lookup_step_export_w##w(int, bool);       \
-  ImportStepFn lookup_import_step_w##w(int, bool);
-LA_DECL_XCH(0) LA_DECL_XCH(1) LA_DECL_XCH(2) LA_DECL_XCH(4) LA_DECL_XCH(8) LA_DECL_XCH(16)
-LA_DECL_XCH(3) LA_DECL_XCH(6) LA_DECL_XCH(12)
-#undef LA_DECL_XCH
-
-StepExportFn lookup_step_export(int W, int gm, bool bf16) {
-  switch (W) {
-    case 1: return lookup_step_export_w1(gm, bf16);
-    case 2: return lookup_step_export_w2(gm, bf16);
-    case 4: return lookup_step_export_w4(gm, bf16);
-    case 8: return lookup_step_export_w8(gm, bf16);
-    case 16: return lookup_step_export_w16(gm, bf16);
-    case 3: return lookup_step_export_w3(gm, bf16);
-    case 6: return lookup_step_export_w6(gm, bf16);
-    case 12: return lookup_step_export_w12(gm, bf16);
-    default: return lookup_step_export_w0(gm, bf16);
-  }
-}
-ImportStepFn lookup_import_step(int W, int gm, bool bf16) {
-  switch (W) {
-    case 1: return lookup_import_step_w1(gm, bf16);
-    case 2: return lookup_import_step_w2(gm, bf16);
-    case 4: return lookup_import_step_w4(gm, bf16);
-    case 8: return lookup_import_step_w8(gm, bf16);
-    case 16: return lookup_import_step_w16(gm, bf16);
-    case 3: return lookup_import_step_w3(gm, bf16);
-    case 6: return lookup_import_step_w6(gm, bf16);
-    case 12: return lookup_import_step_w12(gm, bf16);
-    default: return lookup_import_step_w0(gm, bf16);
-  }
-}
-
-ExchangeFn lookup_export_w0();
-ExchangeFn lookup_export_w1();
-ExchangeFn lookup_export_w2();
-ExchangeFn lookup_export_w4();
-ExchangeFn lookup_export_w8();
-ExchangeFn lookup_export_w16();
-ExchangeFn lookup_export_w3();
-ExchangeFn lookup_export_w6();
-ExchangeFn lookup_export_w12();
-
-ExchangeFn lookup_export(int W) {
-  switch (W) {
-    case 1: return lookup_export_w1();
-    case 2: return lookup_export_w2();
-    case 4: return lookup_export_w4();
-    case 8: return lookup_export_w8();
-    case 16: return lookup_export_w16();
-    case 3: return lookup_export_w3();
-    case 6: return lookup_export_w6();
-    case 12: return lookup_export_w12();
-    default: return lookup_export_w0();
-  }
-}
-constexpr int kExchangeVec = 2;  // coordinates per thread in the exchange kernels
+constexpr int kExchangeVec = 2;  // coordinates per thread in the combine kernel
 
 __global__ void la_fill(float* X, float* B2, float* Bs, const float* x0, float b0sq, uint64_t stride,
                         uint64_t n, uint32_t W) {
@@ -418,9 +361,12 @@ double pass_bytes(const la_ctx* c, bool pre, bool step, bool post, int gm) {
   return b;
 }
 
-int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t tp, int gm, const void* gext) {
+// xch: 0 = a pass of the single-GPU path; 1 / 2 = the pass exports to / imports from the exchange
+// buffer of the by-worker sharding (see la_exchange.cuh).
+int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t tp, int gm, const void* gext,
+                 int xch = 0) {
   const la::SweepKernel k =
-      la::lookup_sweep((int)c->W, c->rule, gm, c->bf16 && gm <= la::kGradQuadratic, pre, step, post);
+      la::lookup_sweep((int)c->W, c->rule, gm, c->bf16 && gm <= la::kGradQuadratic, pre, step, post, xch);
   la::SweepFn fn = k.fn;
   if (!fn)
     return fail(c, LA_ESTATE, "no kernel for this combination (W=%u rule=%d grad=%d bf16=%d)", c->W, c->rule, gm,
@@ -440,6 +386,7 @@ int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t
   p.warm_up_steps = c->warm_up_steps; p.identical_workers = c->identical ? 1u : 0u;
   p.worker_base = c->worker_base;
   p.eta = c->eta; p.eps = c->eps; p.sigma = c->sigma;
+  p.xch = c->S; p.W_total = c->W_total;
   const unsigned block = la::kBlockThreads;
   const uint64_t ngroups = (c->N + (uint64_t)k.vec - 1) / (uint64_t)k.vec;
   uint64_t blocks = (ngroups + block - 1) / block;
@@ -450,7 +397,8 @@ int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t
   const int bps = c->blocks_per_sm > 0 ? c->blocks_per_sm : (step ? 96 : 4096);
   const uint64_t cap = (uint64_t)c->num_sms * (uint64_t)bps;
   if (blocks > cap) blocks = cap;
-  const int cls = !step ? kClassSync : (post ? kClassStepSync : (pre ? kClassSyncStep : kClassLocal));
+  int cls = !step ? kClassSync : (post ? kClassStepSync : (pre ? kClassSyncStep : kClassLocal));
+  if (xch != 0) cls = step ? kClassFused : kClassOther;  // exchange passes: aggregate classes only
   EventPair ep{};
   if (c->profiling) {
     int rc = begin_timed(c, cls, &ep);
@@ -462,13 +410,17 @@ int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t
     LA_CUDA(c, cudaEventRecord(ep.b, c->stream));
     c->pending.push_back(ep);
   }
-  const double bytes = pass_bytes(c, pre, step, post, gm);
+  double bytes = pass_bytes(c, pre, step, post, gm);
+  const double rw = 8.0 * c->W * (double)c->N, ex = 8.0 * (double)c->N;  // replicas one way; the exchange buffer
+  if (xch == 1) bytes += ex - rw - (post ? 4.0 * (double)c->N : 0.0);    // sums stored instead of W means (and no Bs)
+  if (xch == 2) bytes += ex - rw;                                        // totals read instead of W replicas
   if (cls == kClassLocal) { c->stats.launches_local++; c->stats.bytes_local += bytes; }
   else if (cls == kClassSync) { c->stats.launches_sync++; c->stats.bytes_sync += bytes; }
+  else if (cls == kClassOther) { c->stats.launches_other++; }
   else {
     c->stats.launches_fused++; c->stats.bytes_fused += bytes;
     if (cls == kClassStepSync) { c->stats.launches_step_sync++; c->stats.bytes_step_sync += bytes; }
-    else { c->stats.launches_sync_step++; c->stats.bytes_sync_step += bytes; }
+    else if (cls == kClassSyncStep) { c->stats.launches_sync_step++; c->stats.bytes_sync_step += bytes; }
   }
   return LA_OK;
 }
@@ -1120,50 +1072,32 @@ int la_comm_open_peer(la_ctx* c, uint32_t peer_rank, const void* handle64) {
   return LA_OK;
 }
 
-static int exchange_params(la_ctx* c, la::ExchangeParams* p, bool need_peers) {
-  if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
-  std::memset(p, 0, sizeof *p);
-  for (uint32_t r = 0; r < c->world; ++r) {
-    if (need_peers && !c->peerS[r]) return fail(c, LA_ESTATE, "exchange buffer of rank %u not attached", r);
-    p->S[r] = c->peerS[r];
-  }
-  p->X = c->X; p->B2 = c->B2; p->Bs = c->Bs;
-  p->n = c->N; p->stride = c->stride;
-  const uint64_t units = c->stride / 64;
-  p->slice_lo = units * c->rank / c->world * 64;
-  p->slice_hi = units * (c->rank + 1) / c->world * 64;
-  p->W = c->W; p->W_total = c->W_total; p->rank = c->rank; p->world = c->world;
-  return LA_OK;
-}
-
-static unsigned exchange_grid(const la_ctx* c, uint64_t coords) {
-  const uint64_t groups = (coords + kExchangeVecHost - 1) / kExchangeVecHost;
-  uint64_t blocks = (groups + la::kBlockThreads - 1) / la::kBlockThreads;
-  const uint64_t cap = (uint64_t)c->num_sms * 4096;
-  if (blocks > cap) blocks = cap;
-  return blocks ? (unsigned)blocks : 1u;
-}
-
 int la_comm_export(la_ctx* c) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
   DeviceGuard guard(c->device);
-  la::ExchangeParams p;
-  int rc = exchange_params(c, &p, false);
-  if (rc) return rc;
-  la::lookup_export((int)c->W)<<<exchange_grid(c, c->N), la::kBlockThreads, 0, c->stream>>>(p);
-  LA_CUDA(c, cudaGetLastError());
-  c->stats.launches_other++;
-  return LA_OK;
+  return launch_sweep(c, true, false, false, c->t, 0, la::kGradNoise, nullptr, 1);
 }
 
 int la_comm_combine(la_ctx* c) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
   DeviceGuard guard(c->device);
-  la::ExchangeParams p;
-  int rc = exchange_params(c, &p, true);
-  if (rc) return rc;
+  la::CombineParams p{};
+  for (uint32_t r = 0; r < c->world; ++r) {
+    if (!c->peerS[r]) return fail(c, LA_ESTATE, "exchange buffer of rank %u not attached", r);
+    p.S[r] = c->peerS[r];
+  }
+  p.stride = c->stride; p.world = c->world;
+  const uint64_t units = c->stride / 64;
+  p.slice_lo = units * c->rank / c->world * 64;
+  p.slice_hi = units * (c->rank + 1) / c->world * 64;
   if (p.slice_hi > p.slice_lo) {
-    la::la_combine_sums<la::kExchangeVec><<<exchange_grid(c, p.slice_hi - p.slice_lo), la::kBlockThreads, 0, c->stream>>>(p);
+    const uint64_t groups = (p.slice_hi - p.slice_lo) / kExchangeVecHost;
+    uint64_t blocks = (groups + la::kBlockThreads - 1) / la::kBlockThreads;
+    const uint64_t cap = (uint64_t)c->num_sms * 4096;
+    if (blocks > cap) blocks = cap;
+    la::la_combine_sums<la::kExchangeVec><<<(unsigned)blocks, la::kBlockThreads, 0, c->stream>>>(p);
     LA_CUDA(c, cudaGetLastError());
     c->stats.launches_other++;
   }
@@ -1172,55 +1106,20 @@ int la_comm_combine(la_ctx* c) {
 
 int la_comm_import(la_ctx* c) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
   DeviceGuard guard(c->device);
-  la::ExchangeParams p;
-  int rc = exchange_params(c, &p, false);
+  int rc = launch_sweep(c, true, false, false, c->t, 0, la::kGradNoise, nullptr, 2);
   if (rc) return rc;
-  la::la_import_means<la::kExchangeVec><<<exchange_grid(c, c->N), la::kBlockThreads, 0, c->stream>>>(p);
-  LA_CUDA(c, cudaGetLastError());
-  c->stats.launches_other++;
   c->tp = 0; c->nsync += 1;
   return LA_OK;
-}
-
-// Parameters of a step launched outside launch_sweep (the exchange-fused steps).
-static void step_params(const la_ctx* c, la::SweepParams* p, uint64_t t, uint32_t tp, const void* gext, int gm) {
-  std::memset(p, 0, sizeof *p);
-  p->X = c->X; p->B2 = c->B2; p->Bs = c->Bs;
-  p->a = c->pa; p->c = c->pc; p->s = c->has_s ? c->ps : nullptr;
-  p->gext = gext;
-  if (gext) {
-    const uint64_t elem = (gm == la::kGradExternalBF16) ? 2 : 4;
-    p->gext_vec = (c->N % kExchangeVecHost == 0 && (reinterpret_cast<uintptr_t>(gext) % (kExchangeVecHost * elem)) == 0) ? 1u : 0u;
-  }
-  p->n = c->N; p->stride = c->stride; p->j_base = c->j_base;
-  p->seed = c->seed; p->t = t; p->W = c->W; p->tp = tp;
-  p->warm_up_steps = c->warm_up_steps; p->identical_workers = c->identical ? 1u : 0u;
-  p->worker_base = c->worker_base;
-  p->eta = c->eta; p->eps = c->eps; p->sigma = c->sigma;
-}
-
-static unsigned step_grid(const la_ctx* c) {
-  const uint64_t groups = (c->N + kExchangeVecHost - 1) / kExchangeVecHost;
-  uint64_t blocks = (groups + la::kBlockThreads - 1) / la::kBlockThreads;
-  const uint64_t cap = (uint64_t)c->num_sms * (uint64_t)(c->blocks_per_sm > 0 ? c->blocks_per_sm : 96);
-  if (blocks > cap) blocks = cap;
-  return blocks ? (unsigned)blocks : 1u;
 }
 
 static int step_export_impl(la_ctx* c, int gm, const void* gext) {
   if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
   if (c->rule != LA_RULE_ADAALTER) return fail(c, LA_ESTATE, "sharding by worker is implemented for Local AdaAlter only");
-  const bool bf16 = c->bf16 && gm <= la::kGradQuadratic;
-  la::StepExportFn fn = la::lookup_step_export((int)c->W, gm, bf16);
-  if (!fn) return fail(c, LA_ESTATE, "no step+export kernel for this combination (W=%u grad=%d)", c->W, gm);
   DeviceGuard guard(c->device);
-  la::SweepParams p;
-  step_params(c, &p, c->t + 1, c->tp + 1, gext, gm);
-  fn<<<step_grid(c), la::kBlockThreads, 0, c->stream>>>(p, c->S);
-  LA_CUDA(c, cudaGetLastError());
-  c->stats.launches_fused++;
-  c->stats.bytes_fused += 8.0 * c->W * (double)c->N + pass_bytes(c, false, true, false, gm) - 16.0 * c->W * (double)c->N + 8.0 * (double)c->N;
+  int rc = launch_sweep(c, false, true, true, c->t + 1, c->tp + 1, gm, gext, 1);
+  if (rc) return rc;
   c->t += 1; c->tp += 1;
   return LA_OK;
 }
@@ -1241,16 +1140,9 @@ int la_comm_import_step(la_ctx* c) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
   if (c->rule != LA_RULE_ADAALTER) return fail(c, LA_ESTATE, "sharding by worker is implemented for Local AdaAlter only");
-  const bool bf16 = c->bf16 && c->grad_kind <= la::kGradQuadratic;
-  la::ImportStepFn fn = la::lookup_import_step((int)c->W, c->grad_kind, bf16);
-  if (!fn) return fail(c, LA_ESTATE, "no import+step kernel for this combination (W=%u grad=%d)", c->W, c->grad_kind);
   DeviceGuard guard(c->device);
-  la::SweepParams p;
-  step_params(c, &p, c->t + 1, 1u, nullptr, c->grad_kind);
-  fn<<<step_grid(c), la::kBlockThreads, 0, c->stream>>>(p, c->S, c->W_total);
-  LA_CUDA(c, cudaGetLastError());
-  c->stats.launches_fused++;
-  c->stats.bytes_fused += pass_bytes(c, true, true, false, c->grad_kind) - 8.0 * c->W * (double)c->N + 8.0 * (double)c->N;
+  int rc = launch_sweep(c, true, true, false, c->t + 1, 1u, c->grad_kind, nullptr, 2);
+  if (rc) return rc;
   c->nsync += 1; c->t += 1; c->tp = 1;
   return LA_OK;
 }

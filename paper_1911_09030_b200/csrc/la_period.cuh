@@ -35,7 +35,10 @@ template <int W_, int V, int GM, bool BF16, bool POST, int MINB>
 __global__ void __launch_bounds__(LA_PERIOD_BLOCK, MINB) la_period(const PeriodParams pp) {
   const SweepParams& p = pp.base;
   constexpr bool kNeedsNoise = (GM == kGradNoise || GM == kGradNoiseScaled || GM == kGradQuadratic);
-  constexpr int CH = (W_ > 0) ? (W_ < LA_PERIOD_CH ? W_ : LA_PERIOD_CH) : 4;
+  // replicas per chunk: eight where W is a multiple of eight (not for the bf16 variants, which
+  // would spill with eight chains in flight), four otherwise
+  constexpr int kChunkMax = (W_ % 8 == 0 && !BF16) ? LA_PERIOD_CH : (LA_PERIOD_CH < 4 ? LA_PERIOD_CH : 4);
+  constexpr int CH = (W_ > 0) ? (W_ < kChunkMax ? W_ : kChunkMax) : 4;
   constexpr int kOuterUnroll = (W_ > 0) ? kMaxWorkers : 1;
   const uint32_t W = (W_ > 0) ? (uint32_t)W_ : p.W;
   const uint32_t h = pp.h;

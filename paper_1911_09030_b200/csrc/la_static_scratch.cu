@@ -12,7 +12,7 @@
 #include <mutex>
 
 #include "../../include/local_adaalter.h"
-#include "la_exchange.cuh"
+#include "la_sweep.cuh"
 
 namespace {
 
@@ -67,17 +67,19 @@ extern "C" int la_replica_means_static(const float* x_dev, const float* b2_dev, 
   }
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  la::ExchangeParams p{};
-  p.S[0] = scratch;
-  p.X = const_cast<float*>(x_dev);  // the export kernel only reads the replicas
+  // the export pass of the by-worker synchronisation: tree sums over the replicas -> scratch
+  const la::SweepKernel k = la::lookup_sweep((int)W, 0, la::kGradNoise, false, true, false, false, 1);
+  if (!k.fn) return LA_ESTATE;
+  la::SweepParams p{};
+  p.X = const_cast<float*>(x_dev);  // the export pass only reads the replicas
   p.B2 = const_cast<float*>(b2_dev);
-  p.Bs = nullptr;
+  p.xch = scratch;
   p.n = n; p.stride = stride;
-  p.W = W; p.W_total = W; p.rank = 0; p.world = 1;
+  p.W = W; p.W_total = W;
   const unsigned block = la::kBlockThreads;
-  uint64_t blocks = ((n + 1) / 2 + block - 1) / block;
+  uint64_t blocks = ((n + (uint64_t)k.vec - 1) / (uint64_t)k.vec + block - 1) / block;
   if (blocks > (1u << 20)) blocks = 1u << 20;
-  la::lookup_export((int)W)<<<(unsigned)blocks, block, 0, st>>>(p);   // sums -> scratch[0..n), scratch[stride..stride+n)
+  k.fn<<<(unsigned)blocks, block, 0, st>>>(p);   // sums -> scratch[0..n), scratch[stride..stride+n)
   if (cudaGetLastError() != cudaSuccess) return LA_ECUDA;
   uint64_t blocks2 = (n + block - 1) / block;
   if (blocks2 > (1u << 20)) blocks2 = 1u << 20;

@@ -15,6 +15,13 @@
 //   K2 = PRE             stand-alone synchronisation
 //   K3 = STEP+POST       step t'=H fused with its synchronisation
 //   K4 = PRE+STEP        synchronisation fused into the first step of the next period
+// and, when the workers are spread over several GPUs, the same passes cut at the exchange:
+//   XCH = 1 (export)     the adjacent-pair tree SUMS over the local replicas go to the exchange
+//                        buffer instead of the means going back to the replicas
+//                        (PRE: export of the stored replicas; STEP+POST: of this step's y, A^2)
+//   XCH = 2 (import)     the read side is the exchange buffer holding the totals over all ranks
+//                        (one "replica" of sums); means = totals / W_total go to every local replica
+//                        (PRE: plain import; PRE+STEP: import and the first step of the next period)
 #pragma once
 #include <cuda_runtime.h>
 #include <cstdint>
@@ -55,6 +62,8 @@ struct SweepParams {
   uint32_t identical_workers;
   uint32_t worker_base;  // global index of local replica 0 (sharding by worker); keys use worker_base + i
   float eta, eps, sigma;
+  float* xch;            // exchange buffer [2][stride] (sums of x, sums of B^2); XCH kernels only
+  uint32_t W_total;      // workers over all ranks; divisor of the imported totals
 };
 
 __device__ __forceinline__ uint64_t step_index(const SweepParams& p) {
@@ -428,15 +437,21 @@ __device__ __forceinline__ void apply(const Vec<V>& r, const Vec<V>& g, Vec<V>& 
 
 // ACC = true: Algorithm 3 (Local AdaAlter).  ACC = false: Algorithm 2 (Local SGD) — the same sweep
 // without accumulators: y = x - eta_t G, and the synchronisation averages x only.
-template <int W_, int V, int GM, bool BF16, bool PRE, bool STEP, bool POST, int MINB, bool ACC = true>
+template <int W_, int V, int GM, bool BF16, bool PRE, bool STEP, bool POST, int MINB, bool ACC = true, int XCH = 0>
 __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) {
   static_assert(!(PRE && POST), "one synchronisation per pass");
   static_assert(V == 2 || V == 4, "a thread owns 2 or 4 coordinates");
+  static_assert(XCH == 0 || ACC, "the exchange carries x and B^2: Local AdaAlter only");
+  static_assert(XCH != 1 || POST || (PRE && !STEP), "export: sums of a step's results or of the stored replicas");
+  static_assert(XCH != 2 || PRE, "import: the averaged state is what the pass starts from");
+  constexpr bool kExport = (XCH == 1), kImport = (XCH == 2);
   constexpr bool kNeedsNoise = STEP && (GM == kGradNoise || GM == kGradNoiseScaled || GM == kGradQuadratic);
-  constexpr int CH = (W_ > 0) ? (W_ < LA_CH ? W_ : LA_CH) : 4;  // replicas loaded before any is consumed
-  constexpr int kOuterUnroll = (W_ > 0) ? kMaxWorkers : 1;  // static W: unroll fully, so that the
-                                                             // reduction stack is indexed by constants
+  constexpr int WR_ = kImport ? 1 : W_;  // replicas on the READ side (import: the one row of totals)
+  constexpr int CH = (WR_ > 0) ? (WR_ < LA_CH ? WR_ : LA_CH) : 4;  // replicas loaded before any is consumed
+  constexpr int kReadUnroll = (WR_ > 0) ? kMaxWorkers : 1;  // static counts: unroll fully, so that the
+  constexpr int kWriteUnroll = (W_ > 0) ? kMaxWorkers : 1;  // reduction stack is indexed by constants
   const uint32_t W = (W_ > 0) ? (uint32_t)W_ : p.W;
+  const uint32_t Wr = kImport ? 1u : W;
 
   __shared__ uint64_t keys[kMaxWorkers];
   if (kNeedsNoise) {
@@ -469,6 +484,10 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
   const uint64_t x_base = reinterpret_cast<uint64_t>(p.X);
   const uint64_t b_delta = reinterpret_cast<uint64_t>(p.B2) - x_base;
   const uint64_t stride_bytes = p.stride * sizeof(float);
+  // read side: the replicas, or (import) the exchange buffer seen as one replica whose "B^2"
+  // sits one stride after its "x"
+  const uint64_t rd_base = kImport ? reinterpret_cast<uint64_t>(p.xch) : x_base;
+  const uint64_t rd_b_delta = kImport ? stride_bytes : b_delta;
 
   constexpr bool kExternal = STEP && (GM == kGradExternalF32 || GM == kGradExternalBF16);
   constexpr uint64_t kGradElem = (GM == kGradExternalBF16) ? 2 : 4;
@@ -479,9 +498,9 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
   GradChunk<V, kExternal ? CH : 1> gnxt;
   CoordInputs<V> in_next;
   load_coord<GM, STEP, kLoadsBs, V>(in_next, p, grp * V);
-  uint64_t ld_addr = x_base + grp * (V * sizeof(float));
+  uint64_t ld_addr = rd_base + grp * (V * sizeof(float));
   uint64_t g_addr = g_base + grp * (V * kGradElem);
-  load_chunk<V, CH, ACC>(nxt, ld_addr, b_delta, stride_bytes, W, 0u);
+  load_chunk<V, CH, ACC>(nxt, ld_addr, rd_b_delta, stride_bytes, Wr, 0u);
   if (kExternal) load_grads<GM, V, kExternal ? CH : 1>(gnxt, p, g_addr, g_row_bytes, W, 0u, grp * V);
 
   for (;;) {
@@ -495,19 +514,19 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
     Vec<V> r;
     if (kLoadsBs) r = step_size<V>(in.bs, q, eta_t);
     if (!ACC) r = splat<V>(eta_t);
-    typename TreeFor<W_, V, ACC>::type tree;
+    typename TreeFor<WR_, V, ACC>::type tree;
 
-#pragma unroll kOuterUnroll
-    for (uint32_t i0 = 0; i0 < W; i0 += CH) {
+#pragma unroll kReadUnroll
+    for (uint32_t i0 = 0; i0 < Wr; i0 += CH) {
       ReplicaChunk<V, CH> cur = nxt;
       GradChunk<V, kExternal ? CH : 1> gcur = gnxt;
-      if (i0 + CH < W) {
-        load_chunk<V, CH, ACC>(nxt, ld_addr, b_delta, stride_bytes, W, i0 + CH);
+      if (i0 + CH < Wr) {
+        load_chunk<V, CH, ACC>(nxt, ld_addr, rd_b_delta, stride_bytes, Wr, i0 + CH);
         if (kExternal) load_grads<GM, V, kExternal ? CH : 1>(gnxt, p, g_addr, g_row_bytes, W, i0 + CH, off);
       } else if (has_next) {
         load_coord<GM, STEP, kLoadsBs, V>(in_next, p, next_grp * V);
-        ld_addr = x_base + next_grp * (V * sizeof(float));
-        load_chunk<V, CH, ACC>(nxt, ld_addr, b_delta, stride_bytes, W, 0u);
+        ld_addr = rd_base + next_grp * (V * sizeof(float));
+        load_chunk<V, CH, ACC>(nxt, ld_addr, rd_b_delta, stride_bytes, Wr, 0u);
         if (kExternal) {
           g_addr = g_base + next_grp * (V * kGradElem);
           load_grads<GM, V, kExternal ? CH : 1>(gnxt, p, g_addr, g_row_bytes, W, 0u, next_grp * V);
@@ -516,16 +535,16 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
       asm volatile("" ::: "memory");
 #pragma unroll
       for (int k = 0; k < CH; ++k)
-        if (i0 + k < W) {
+        if (i0 + k < Wr) {
           const uint32_t i = i0 + k;
           if (PRE) {
-            tree.push_in_chunk(i, k, i0 + CH <= W, cur.x[k], cur.b[k]);
+            tree.push_in_chunk(i, k, i0 + CH <= Wr, cur.x[k], cur.b[k]);
           } else {
             const Vec<V> g = kExternal ? gcur.g[kExternal ? k : 0]
                                        : gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
             apply<V, ACC>(r, g, cur.x[k], cur.b[k]);
             if (POST) {
-              tree.push_in_chunk(i, k, i0 + CH <= W, cur.x[k], cur.b[k]);
+              tree.push_in_chunk(i, k, i0 + CH <= Wr, cur.x[k], cur.b[k]);
             } else {
               store_replica<V, ACC>(st_addr, b_delta, stride_bytes, cur.x[k], cur.b[k]);
             }
@@ -534,28 +553,34 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
     }
 
     if (PRE || POST) {
-      // synchronisation branch of Algorithm 3: means over workers; the mean accumulator is
-      // also the new stale denominator
       tree.finish();
-      const Vec<V> xm = div_by_workers<W_, V>(tree.x[0], W);
-      Vec<V> bm = xm;
-      if (ACC) {
-        bm = div_by_workers<W_, V>(tree.b[0], W);
-        st_stream<V>(p.Bs + off, bm);
-      }
-      if (PRE && STEP) {
-        // first step of the next period: every replica starts from the mean, t' = 1
-        if (ACC) r = step_size<V>(bm, q, eta_t);
-#pragma unroll kOuterUnroll
-        for (uint32_t i = 0; i < W; ++i) {
-          Vec<V> xv = xm, bv = bm;
-          const Vec<V> g = gradient<GM, BF16, V>(p, in, xv, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
-          apply<V, ACC>(r, g, xv, bv);
-          store_replica<V, ACC>(st_addr, b_delta, stride_bytes, xv, bv);
-        }
+      if (kExport) {
+        // the means are formed after the exchange, from the totals over all ranks
+        st_stream<V>(p.xch + off, tree.x[0]);
+        st_stream<V>(p.xch + p.stride + off, tree.b[0]);
       } else {
-#pragma unroll kOuterUnroll
-        for (uint32_t i = 0; i < W; ++i) store_replica<V, ACC>(st_addr, b_delta, stride_bytes, xm, bm);
+        // synchronisation branch of Algorithm 3: means over workers; the mean accumulator is
+        // also the new stale denominator
+        const Vec<V> xm = kImport ? div_by_workers<0, V>(tree.x[0], p.W_total) : div_by_workers<W_, V>(tree.x[0], W);
+        Vec<V> bm = xm;
+        if (ACC) {
+          bm = kImport ? div_by_workers<0, V>(tree.b[0], p.W_total) : div_by_workers<W_, V>(tree.b[0], W);
+          st_stream<V>(p.Bs + off, bm);
+        }
+        if (PRE && STEP) {
+          // first step of the next period: every replica starts from the mean, t' = 1
+          if (ACC) r = step_size<V>(bm, q, eta_t);
+#pragma unroll kWriteUnroll
+          for (uint32_t i = 0; i < W; ++i) {
+            Vec<V> xv = xm, bv = bm;
+            const Vec<V> g = gradient<GM, BF16, V>(p, in, xv, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
+            apply<V, ACC>(r, g, xv, bv);
+            store_replica<V, ACC>(st_addr, b_delta, stride_bytes, xv, bv);
+          }
+        } else {
+#pragma unroll kWriteUnroll
+          for (uint32_t i = 0; i < W; ++i) store_replica<V, ACC>(st_addr, b_delta, stride_bytes, xm, bm);
+        }
       }
     }
     if (!has_next) break;
@@ -629,6 +654,7 @@ struct SweepKernel {
   int vec;
 };
 // rule: 0 = Local AdaAlter, 1 = Local SGD, 2 = Distributed AdaGrad (one kernel per step)
-SweepKernel lookup_sweep(int W, int rule, int gm, bool bf16, bool pre, bool step, bool post);
+// xch: 0 = single-GPU pass, 1 = export to / 2 = import from the exchange buffer (rule 0 only)
+SweepKernel lookup_sweep(int W, int rule, int gm, bool bf16, bool pre, bool step, bool post, int xch = 0);
 
 }  // namespace la
