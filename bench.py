@@ -427,6 +427,8 @@ def run_ours(args, wl):
         if wl.name != "c2":
             extras["c2"] = side_config(la, workloads.config("c2"), peak, barrier, sampler)
         extras["c4_sync_period_sweep"] = sync_period_sweep(la, workloads.config("c4"), peak, barrier)
+        # the by-worker layout with this one rank (exchange kernels and host-ordered phases included)
+        extras["by_worker"] = by_worker_leg(la, workloads.config("c2"), dd, rank, world, barrier, T=64)
 
     if rank == 0:
         sampler.stop()
@@ -520,6 +522,91 @@ def sync_period_sweep(la, wl, peak, barrier):
     return {"workload": workload_config(wl, None)["workload"].split(", H=")[0], "unit": UNIT, "rows": rows}
 
 
+def by_worker_leg(la, wl, dd, rank, world, barrier, T=None, periods=(1, 4, 16), exchanges=("peer", "allreduce")):
+    """Sharding BY WORKER (the paper's layout, Section 4.2): every rank holds wl.W replicas of the
+    W_total = wl.W x world workers and the ranks exchange x and B^2 every H steps — export of the
+    local tree sums, exchange (peer-load combine kernel, or an all-reduce of the buffer by
+    torch.distributed), import; the steps next to a synchronisation are fused with it.  Times T
+    iterations per (H, exchange): whole-job rate, host time per exchange and its share."""
+    import torch
+    from paper_1911_09030_b200 import sharding
+    from paper_1911_09030_b200.worker_sharded import CudaEngine, WorkerShardedJob
+    T = int(T or wl.T)
+    arr = wl.arrays()
+    rows = []
+    for H in periods:
+        for exch in exchanges:
+            ctx = la.LocalAdaAlter.with_torch_arena(wl.sizes, wl.W, wl.eta, wl.eps, la.LA_H_NEVER, b0sq=wl.b0sq)
+            if wl.grad == "quadratic":
+                ctx.set_grad_quadratic(wl.noise_seed, arr["a"], arr["c"], wl.sigma)
+            elif wl.grad == "noise_scaled":
+                ctx.set_grad_noise(wl.noise_seed, arr["s"])
+            else:
+                ctx.set_grad_noise(wl.noise_seed, None)
+            if wl.bf16_grads:
+                ctx.set_grad_dtype(la.LA_BF16)
+            eng = CudaEngine(ctx, rank, world)
+            if dd is not None and exch == "peer":
+                eng.attach_peers(dd)
+            job = WorkerShardedJob(eng, H, exchange=exch, dist=dd, fused=True)
+            job.run(2 * H if 2 * H < T else T)          # warm-up: two periods
+            barrier()
+            job.exchange_seconds, syncs0 = 0.0, job.syncs
+            t0 = time.perf_counter()
+            job.run(T)
+            barrier()
+            sec = sharding.max_over_ranks(time.perf_counter() - t0, dd)
+            exs = sharding.max_over_ranks(job.exchange_seconds, dd)
+            nsync = job.syncs - syncs0
+            rows.append({"H": H, "exchange": exch, "T": T, "syncs": nsync, "ms_per_iteration": 1e3 * sec / T,
+                         "value": wl.W * world * wl.N * T / sec,
+                         "exchange_ms_per_sync": 1e3 * exs / nsync if nsync else None,
+                         "exchange_share_of_time": exs / sec,
+                         "exchange_bytes_per_rank_per_sync": 8 * wl.N})
+            ctx.close()
+            torch.cuda.empty_cache()
+    return {"sharding": "by worker: %d local replicas per rank, W_total = %d" % (wl.W, wl.W * world),
+            "workload": workload_config(wl, None)["workload"], "unit": UNIT, "ranks": world,
+            "exchange_fused_steps": True, "rows": rows}
+
+
+def run_by_worker(args, wl):
+    """`--sharding worker`: the by-worker layout alone, one JSON line."""
+    import torch
+    import torch.distributed as dist
+    from paper_1911_09030_b200 import local_adaalter as la
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    use_dist = world > 1 or ("RANK" in os.environ and "MASTER_PORT" in os.environ)
+    if use_dist:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        # keep the communicator's own log lines (ranks, transports) on stderr, next to the numbers
+        os.environ.setdefault("NCCL_DEBUG", "INFO")
+        os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+        os.environ.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dd = dist if use_dist else None
+
+    def barrier():
+        if use_dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    doc = by_worker_leg(la, wl, dd, rank, world, barrier, T=args.T)
+    if rank == 0:
+        best = max(doc["rows"], key=lambda r: r["value"])
+        line = {"metric": METRIC, "value": best["value"], "unit": UNIT, "n_gpus": world, "steps": 1, "warmup": 1,
+                "ms_per_step": best["ms_per_iteration"] * best["T"], "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": dict(workload_config(wl, args), sharding=doc["sharding"], H=best["H"], exchange=best["exchange"]),
+                "by_worker": doc}
+        print(json.dumps(line), flush=True)
+    if use_dist:
+        dist.destroy_process_group()
+
+
 def run_report(args):
     """All five configurations plus the synchronisation-period sweep of configuration 4
     (H in {1,4,16,64} x {unfused, step+sync, sync+step, temporal blocking}): per-kernel-class device time, GB/s
@@ -608,6 +695,71 @@ def run_report(args):
               f"{f2(r['us_fused'], 1)} ({f2(r['GBps_fused'])}) | {f2(100 * r['sync_share_of_time'], 1)} % |")
 
 
+def run_kernel_report(args):
+    """Per-kernel GB/s away from the benchmark configurations: worker counts with their own
+    instantiation (3, 6, 12), worker counts known only at run time (5, 24, 32, 64), and
+    caller-supplied gradient tables in fp32 and bf16 (W = 4, 8, 16).  N = 2^24, pure-noise gradients
+    (the shape of configuration 4), every pass timed by CUDA events around the launch.
+    Markdown table to stdout, JSON to --report-out."""
+    import torch
+    from paper_1911_09030_b200 import local_adaalter as la
+    torch.cuda.set_device(0)
+    peak, peak_kind = measured_peak()
+    N = args.N or (1 << 24)
+    rows = []
+
+    def classes(ctx, W, what):
+        st = ctx.get_stats(reset=True)
+        for cls in ("local", "sync", "step_sync", "sync_step"):
+            n = st[f"launches_{cls}"]
+            if n and st[f"ms_{cls}"] > 0:
+                ms = st[f"ms_{cls}"] / n
+                gbs = st[f"bytes_{cls}"] / n / (ms * 1e-3) / 1e9
+                rows.append({"W": W, "gradients": what, "kernel": KERNEL_NAMES[cls], "launches": int(n),
+                             "us_per_launch": 1e3 * ms, "GBps": gbs, "frac": gbs / peak})
+
+    for W in args.workers:
+        ctx = la.LocalAdaAlter.with_torch_arena([N], W, 0.01, 1e-2, 4)
+        ctx.set_grad_noise(4, None)
+        for fusion in (la.LA_FUSE_NONE, la.LA_FUSE_STEP_SYNC, la.LA_FUSE_SYNC_STEP):
+            ctx.set_fusion(fusion)
+            ctx.run(8)
+        ctx.sync_stream()
+        ctx.get_stats(reset=True)
+        ctx.set_profiling(True)
+        for fusion in (la.LA_FUSE_NONE, la.LA_FUSE_STEP_SYNC, la.LA_FUSE_SYNC_STEP):
+            ctx.set_fusion(fusion)
+            ctx.run(24)
+        ctx.set_profiling(False)
+        classes(ctx, W, "generated (noise)")
+        if W in args.table_workers:
+            for dtype, name, tdt in ((la.LA_F32, "fp32 table", torch.float32), (la.LA_BF16, "bf16 table", torch.bfloat16)):
+                G = torch.randn(W, N, device="cuda", dtype=torch.float32).to(tdt)
+                ctx.set_fusion(la.LA_FUSE_STEP_SYNC)
+                for _ in range(8):
+                    ctx.step_grads(G.data_ptr(), dtype)
+                ctx.sync_stream()
+                ctx.get_stats(reset=True)
+                ctx.set_profiling(True)
+                for _ in range(24):
+                    ctx.step_grads(G.data_ptr(), dtype)
+                ctx.set_profiling(False)
+                classes(ctx, W, name)
+                del G
+        ctx.close()
+        torch.cuda.empty_cache()
+    doc = {"N": N, "peak_GBps": peak, "peak_kind": peak_kind, "rows": rows}
+    if args.report_out:
+        os.makedirs(os.path.dirname(os.path.abspath(args.report_out)), exist_ok=True)
+        with open(args.report_out, "w") as f:
+            json.dump(doc, f, indent=1)
+    print(f"| W | gradients | kernel | launches | us per launch | GB/s | of {peak:.0f} ({peak_kind}) |")
+    print("|---|---|---|---|---|---|---|")
+    for r in rows:
+        print(f"| {r['W']} | {r['gradients']} | {r['kernel']} | {r['launches']} | {r['us_per_launch']:.1f} | "
+              f"{r['GBps']:.0f} | {r['frac']:.3f} |")
+
+
 def run_tradeoff(args):
     """Single-GPU analogue of the paper's Table 2 (quality and time against the synchronisation
     period): the noisy quadratic of configuration 3 at N = 2^24, T = 256 iterations, for Local
@@ -670,6 +822,9 @@ def main():
     ap.add_argument("--N", type=int, default=None, help="override the size (one flat tensor), e.g. for small ncu captures")
     ap.add_argument("--fusion", type=int, default=1, help="0 unfused, 1 step+sync, 2 sync+next step")
     ap.add_argument("--blocks-per-sm", type=int, default=0)
+    ap.add_argument("--sharding", default="coordinate", choices=["coordinate", "worker"],
+                    help="coordinate: every rank owns a coordinate range, no collective (the headline); "
+                         "worker: every rank owns W replicas and the ranks exchange x, B^2 every H steps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-period", action="store_true", help="skip the extra temporal-blocking measurement")
     ap.add_argument("--main-only", action="store_true",
@@ -677,6 +832,10 @@ def main():
     ap.add_argument("--report", action="store_true", help="all configurations + the H sweep (not the JSON line)")
     ap.add_argument("--report-out", default=None)
     ap.add_argument("--tradeoff", action="store_true", help="quality/time against H on a noisy quadratic (table)")
+    ap.add_argument("--report-kernels", action="store_true",
+                    help="per-kernel GB/s for worker counts and gradient tables outside the five configurations")
+    ap.add_argument("--workers", type=lambda v: [int(x) for x in v.split(",")], default=[3, 6, 12, 5, 24, 32, 64, 4, 8, 16])
+    ap.add_argument("--table-workers", type=lambda v: [int(x) for x in v.split(",")], default=[4, 8, 16])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -684,6 +843,8 @@ def main():
         return run_report(args)
     if args.tradeoff:
         return run_tradeoff(args)
+    if args.report_kernels:
+        return run_kernel_report(args)
     from paper_1911_09030_b200 import workloads
     wl = workloads.config(args.workload)
     if args.H is not None:
@@ -694,6 +855,8 @@ def main():
         wl.sizes = [args.N]
     if args.impl == "reference":
         run_reference(args, wl)
+    elif args.sharding == "worker":
+        run_by_worker(args, wl)
     else:
         run_ours(args, wl)
 

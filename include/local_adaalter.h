@@ -44,7 +44,8 @@ enum {
   LA_ENOMEM = -2, /* device or host allocation failed, or caller arena too small */
   LA_ECUDA = -3,  /* a CUDA runtime call failed; message in la_last_error */
   LA_ESTATE = -4, /* call not valid in the context's current configuration */
-  LA_ETOOBIG = -5 /* size exceeds a fixed capacity (la_replica_means_static) */
+  LA_ETOOBIG = -5, /* size exceeds a fixed capacity (la_replica_means_static) */
+  LA_EBOUNDS = -6  /* checked build only: a kernel computed an address outside its ranges (skipped, reported) */
 };
 
 enum { LA_F32 = 0, LA_BF16 = 1 };               /* gradient dtype */
@@ -260,6 +261,24 @@ int la_comm_import_step(la_ctx* ctx);
 int la_noise_tables(float* radius_dev, float* cos_dev, float* sin_dev, void* stream);
 /* Block until the context's stream is idle. */
 int la_stream_sync(la_ctx* ctx);
+
+/* ---- checked build ----------------------------------------------------------------------------
+ * (No counterpart in the paper: a development aid.)  liblocal_adaalter_debug.so is the same
+ * library compiled with -DLA_DEBUG.  Its kernels test every global-memory address they form
+ * against the byte ranges the pass may touch (state arena, caller's gradient table, exchange
+ * buffer) and the running row pointers against base + (replica * stride + coordinate) * 4.  An
+ * offending access is skipped (a load yields 0) and counted; nothing traps or asserts.  The next
+ * synchronising call (la_stream_sync, la_read_state / la_read_range, la_get_stats) then returns
+ * LA_EBOUNDS with the first offending address in la_last_error, and clears the count.  The
+ * arithmetic is unchanged (results stay bitwise equal to the normal library); it is slower and is
+ * never the library that is timed.  The kernel that combines the ranks' exchange buffers
+ * (la_comm_combine) is not range-checked.
+ * la_debug_build: 1 in the checked library, 0 in the normal one.
+ * la_debug_narrow: test knob of the checked library (LA_ESTATE in the normal one): the kernels
+ * treat the last `bytes` bytes of the state arena as foreign, so that in-bounds accesses there are
+ * reported and skipped — a way to see the report without forming a bad address.  0 restores. */
+int la_debug_build(void);
+int la_debug_narrow(la_ctx* ctx, uint64_t bytes);
 
 /* ---- for callers that must not allocate ------------------------------------------------------
  * (The paper has no counterpart: this is a deployment variant of the replica average that

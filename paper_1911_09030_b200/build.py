@@ -1,9 +1,10 @@
 """Build the CUDA library in-tree for sm_100a (nvcc cross-compiles without a GPU).
 
-    python -m paper_1911_09030_b200.build [--force]
+    python -m paper_1911_09030_b200.build [--force] [--debug]
 
-Produces `paper_1911_09030_b200/liblocal_adaalter.so`.  Object files go to
-`paper_1911_09030_b200/_build/`.  Device code is compiled with `-fmad=false`: every
+Produces `paper_1911_09030_b200/liblocal_adaalter.so`; with --debug the checked build
+`liblocal_adaalter_debug.so` (the same sources with -DLA_DEBUG: kernels range-check their
+addresses).  Object files go to `paper_1911_09030_b200/_build/` (`_build/debug/`).  Device code is compiled with `-fmad=false`: every
 fused multiply-add in the kernels is written explicitly, none may be introduced.
 """
 from __future__ import annotations
@@ -39,7 +40,10 @@ def _stale(target, inputs):
     return any(os.path.getmtime(p) > t for p in inputs)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    OBJ = os.path.join(HERE, "_build", "debug") if debug else globals()["OBJ"]
+    LIB = os.path.join(HERE, "liblocal_adaalter_debug.so") if debug else globals()["LIB"]
+    FLAGS = globals()["FLAGS"] + (["-DLA_DEBUG"] if debug else [])
     os.makedirs(OBJ, exist_ok=True)
     srcs, deps = _sources(), _deps()
     jobs = []
@@ -71,4 +75,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

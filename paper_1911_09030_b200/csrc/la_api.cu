@@ -103,7 +103,7 @@ __global__ void la_broadcast_replica0(float* X, float* B2, uint64_t stride, uint
 __global__ void la_noise_tables_kernel(float* radius, float* cs, float* sn) {
   const uint32_t nthreads = gridDim.x * blockDim.x;
   for (uint32_t q = blockIdx.x * blockDim.x + threadIdx.x; q < (1u << 24); q += nthreads) {
-    if (radius) radius[q] = radius_from_u24(q + 1u);
+    if (radius) radius[q] = radius_from_top24(q << 8);
     if (cs || sn) {
       float c, s;
       cossin_from_top24(q << 8, c, s);
@@ -211,6 +211,10 @@ struct la_ctx {
   float* peerS[la::kMaxRanks] = {};
   void* ipc_opened[la::kMaxRanks] = {};
   double* diag = nullptr;  // two doubles for la_diagnostics, allocated on its first call
+  // checked build (LA_DEBUG): device status words the kernels report address violations into,
+  // and a test knob that makes the kernels treat the last `dbg_narrow` bytes of the arena as foreign
+  unsigned long long* dbg_status = nullptr;
+  uint64_t dbg_narrow = 0, arena_size = 0;
   // CUDA-graph replay of whole periods (la_set_graph)
   bool use_graph = false, capturing = false;
   uint64_t* sched = nullptr;       // device: global step count before the period being replayed
@@ -326,6 +330,36 @@ int begin_timed(la_ctx* c, int cls, EventPair* ep) {
   return LA_OK;
 }
 
+// ---- checked build ---------------------------------------------------------------------------
+#ifdef LA_DEBUG
+void fill_debug_ranges(const la_ctx* c, la::DebugRanges* d, const void* gext, uint64_t gext_bytes) {
+  const uint64_t a = reinterpret_cast<uint64_t>(c->arena);
+  d->lo[0] = a; d->hi[0] = a + c->arena_size - c->dbg_narrow;
+  d->lo[1] = reinterpret_cast<uint64_t>(gext); d->hi[1] = d->lo[1] + gext_bytes;
+  d->lo[2] = reinterpret_cast<uint64_t>(c->S); d->hi[2] = d->lo[2] + (c->S ? 2 * c->stride * sizeof(float) : 0);
+  d->status = c->dbg_status;
+}
+#endif
+
+// After a synchronising call in the checked build: turn recorded violations into an error.
+int debug_poll(la_ctx* c) {
+#ifdef LA_DEBUG
+  if (!c->dbg_status) return LA_OK;
+  unsigned long long st[3] = {0, 0, 0};
+  LA_CUDA(c, cudaMemcpyAsync(st, c->dbg_status, sizeof st, cudaMemcpyDeviceToHost, c->stream));
+  LA_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (st[0] != 0) {
+    LA_CUDA(c, cudaMemsetAsync(c->dbg_status, 0, sizeof st, c->stream));
+    const char* kind = (st[2] & 0xFF) == 2 ? "is not the row its replica index and coordinate give" : "lies outside every range the pass may touch";
+    return fail(c, LA_EBOUNDS, "checked build: %llu access(es) skipped; the first, at device address 0x%llx (%llu bytes), %s",
+                st[0], st[1], (st[2] >> 8), kind);
+  }
+#else
+  (void)c;
+#endif
+  return LA_OK;
+}
+
 // ---- kernel dispatch ------------------------------------------------------------------------
 // Algorithmic bytes of one pass (what must cross HBM with the thread-per-coordinate mapping):
 // every replica's x and B^2 read and written once, worker-independent arrays once.
@@ -387,6 +421,9 @@ int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t
   p.worker_base = c->worker_base;
   p.eta = c->eta; p.eps = c->eps; p.sigma = c->sigma;
   p.xch = c->S; p.W_total = c->W_total;
+#ifdef LA_DEBUG
+  fill_debug_ranges(c, &p.dbg, gext, gext ? (uint64_t)c->W * c->N * (gm == la::kGradExternalBF16 ? 2u : 4u) : 0u);
+#endif
   const unsigned block = la::kBlockThreads;
   const uint64_t ngroups = (c->N + (uint64_t)k.vec - 1) / (uint64_t)k.vec;
   uint64_t blocks = (ngroups + block - 1) / block;
@@ -442,6 +479,9 @@ int launch_period(la_ctx* c, uint32_t h, bool post) {
   p.worker_base = c->worker_base;
   p.eta = c->eta; p.eps = c->eps; p.sigma = c->sigma;
   pp.h = h;
+#ifdef LA_DEBUG
+  fill_debug_ranges(c, &p.dbg, nullptr, 0);
+#endif
   const unsigned block = (unsigned)k.block;
   const uint64_t ngroups = (c->N + (uint64_t)k.vec - 1) / (uint64_t)k.vec;
   uint64_t blocks = (ngroups + block - 1) / block;
@@ -533,6 +573,7 @@ int la_create_ex(la_ctx** out, const la_config* cfg) {
   auto bail = [&](int code, const char* what, cudaError_t e) {
     fail(nullptr, code, "%s%s%s", what, e != cudaSuccess ? ": " : "", e != cudaSuccess ? cudaGetErrorString(e) : "");
     if (c->owns_arena && c->arena) cudaFree(c->arena);
+    if (c->dbg_status) cudaFree(c->dbg_status);
     delete c;
     return code;
   };
@@ -569,6 +610,16 @@ int la_create_ex(la_ctx** out, const la_config* cfg) {
     }
     c->owns_arena = true;
   }
+  c->arena_size = need;
+#ifdef LA_DEBUG
+  if ((e = cudaMalloc((void**)&c->dbg_status, 4 * sizeof(unsigned long long))) != cudaSuccess) {
+    c->dbg_status = nullptr;
+    cudaGetLastError();
+    return bail(LA_ENOMEM, "cudaMalloc of the checked build's status words failed", e);
+  }
+  if ((e = cudaMemsetAsync(c->dbg_status, 0, 4 * sizeof(unsigned long long), c->stream)) != cudaSuccess)
+    return bail(LA_ECUDA, "cudaMemsetAsync", e);
+#endif
   float* base = (float*)c->arena;
   c->X = base;
   c->B2 = c->X + (uint64_t)c->W * c->stride;
@@ -581,7 +632,7 @@ int la_create_ex(la_ctx** out, const la_config* cfg) {
     return bail(LA_ECUDA, "cudaMemsetAsync", e);
   c->grad_kind = la::kGradNoise;
   rc = do_fill(c, nullptr);
-  if (rc) { g_create_error = c->err; if (c->owns_arena) cudaFree(c->arena); delete c; return rc; }
+  if (rc) { g_create_error = c->err; if (c->owns_arena) cudaFree(c->arena); if (c->dbg_status) cudaFree(c->dbg_status); delete c; return rc; }
   *out = c;
   return LA_OK;
 }
@@ -603,6 +654,7 @@ void la_destroy(la_ctx* c) {
   for (auto*& m : c->ipc_opened) if (m) { cudaIpcCloseMemHandle(m); m = nullptr; }
   if (c->S) cudaFree(c->S);
   if (c->diag) cudaFree(c->diag);
+  if (c->dbg_status) cudaFree(c->dbg_status);
   if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
   if (c->sched) cudaFree(c->sched);
   if (c->owns_arena && c->arena) cudaFree(c->arena);
@@ -942,7 +994,7 @@ int la_read_range(la_ctx* c, uint32_t worker, uint64_t j0, uint64_t n, float* x_
     if (bs_host) LA_CUDA(c, cudaMemcpyAsync(bs_host, c->Bs + j0, bytes, cudaMemcpyDeviceToHost, c->stream));
   }
   LA_CUDA(c, cudaStreamSynchronize(c->stream));
-  return LA_OK;
+  return debug_poll(c);
 }
 
 int la_read_state(la_ctx* c, uint32_t worker, float* x_host, float* b2_host, float* bs_host) {
@@ -996,7 +1048,7 @@ int la_get_stats(la_ctx* c, la_stats* out, int reset) {
   if (rc) return rc;
   *out = c->stats;
   if (reset) c->stats = la_stats{};
-  return LA_OK;
+  return debug_poll(c);
 }
 
 // ---- sharding by worker -------------------------------------------------------------------
@@ -1183,7 +1235,27 @@ int la_stream_sync(la_ctx* c) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   DeviceGuard guard(c->device);
   LA_CUDA(c, cudaStreamSynchronize(c->stream));
+  return debug_poll(c);
+}
+
+int la_debug_build(void) {
+#ifdef LA_DEBUG
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+int la_debug_narrow(la_ctx* c, uint64_t bytes) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+#ifdef LA_DEBUG
+  if (bytes > c->arena_size) return fail(c, LA_EINVAL, "more than the arena holds");
+  c->dbg_narrow = bytes;
   return LA_OK;
+#else
+  (void)bytes;
+  return fail(c, LA_ESTATE, "this is not the checked build (compile with -DLA_DEBUG)");
+#endif
 }
 
 }  // extern "C"

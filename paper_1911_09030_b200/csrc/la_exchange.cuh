@@ -38,6 +38,9 @@ struct CombineParams {
 
 template <int V>
 __global__ void __launch_bounds__(LA_BLOCK) la_combine_sums(const CombineParams p) {
+#ifdef LA_DEBUG
+  dbg_begin(DebugRanges{});  // the ranks' buffers are not range-checked
+#endif
   const uint64_t ngroups = (p.slice_hi - p.slice_lo) / (uint64_t)V;
   const uint64_t nthreads = (uint64_t)gridDim.x * blockDim.x;
   for (uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < ngroups; grp += nthreads) {

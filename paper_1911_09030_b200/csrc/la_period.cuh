@@ -44,6 +44,9 @@ __global__ void __launch_bounds__(LA_PERIOD_BLOCK, MINB) la_period(const PeriodP
   const uint32_t h = pp.h;
 
   // stream keys of every (step, worker) of this pass, and the per-step scalars
+#ifdef LA_DEBUG
+  dbg_begin(p.dbg);
+#endif
   __shared__ uint64_t keys[kPeriodMax][kMaxWorkers];
   __shared__ float eta_s[kPeriodMax], q_s[kPeriodMax];
   __shared__ Vec<V> r_s[kPeriodMax][LA_PERIOD_BLOCK];
@@ -94,7 +97,7 @@ __global__ void __launch_bounds__(LA_PERIOD_BLOCK, MINB) la_period(const PeriodP
 #pragma unroll kOuterUnroll
     for (uint32_t i0 = 0; i0 < W; i0 += CH) {
       ReplicaChunk<V, CH> cur;
-      load_chunk<V, CH>(cur, ld_addr, b_delta, stride_bytes, W, i0);
+      load_chunk<V, CH>(cur, ld_addr, b_delta, stride_bytes, W, i0 LA_DBG_ARG(x_base + off * sizeof(float)));
       // steps outside, the chunk's replicas inside: CH independent gradient chains per iteration
 #pragma unroll kPeriodUnroll
       for (uint32_t s = 0; s < h; ++s) {
@@ -113,7 +116,8 @@ __global__ void __launch_bounds__(LA_PERIOD_BLOCK, MINB) la_period(const PeriodP
           if (POST) {
             tree.push_in_chunk(i0 + k, k, i0 + CH <= W, cur.x[k], cur.b[k]);
           } else {
-            store_replica<V>(st_addr, b_delta, stride_bytes, cur.x[k], cur.b[k]);
+            store_replica<V>(st_addr, b_delta, stride_bytes, cur.x[k], cur.b[k]
+                             LA_DBG_ARG(x_base + off * sizeof(float) + (uint64_t)(i0 + k) * stride_bytes));
           }
         }
     }
@@ -123,7 +127,8 @@ __global__ void __launch_bounds__(LA_PERIOD_BLOCK, MINB) la_period(const PeriodP
       const Vec<V> bm = div_by_workers<W_, V>(tree.b[0], W);
       st_stream<V>(p.Bs + off, bm);
 #pragma unroll kOuterUnroll
-      for (uint32_t i = 0; i < W; ++i) store_replica<V>(st_addr, b_delta, stride_bytes, xm, bm);
+      for (uint32_t i = 0; i < W; ++i)
+        store_replica<V>(st_addr, b_delta, stride_bytes, xm, bm LA_DBG_ARG(x_base + off * sizeof(float) + (uint64_t)i * stride_bytes));
     }
   }
 }

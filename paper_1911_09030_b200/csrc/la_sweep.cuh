@@ -40,7 +40,54 @@ enum GradKind : int {
   kGradExternalBF16 = 5  // g read from a [W][N] bf16 table
 };
 
+// Checked build (compile with -DLA_DEBUG; a separate library, never the one that is timed).
+// compute-sanitizer's job, done by the kernels themselves: every global access is tested against
+// the byte ranges the pass may touch, and the running row pointers against the closed form
+// base + (replica * stride + coordinate) * 4.  A violation is counted in a status word that the
+// host reads at the next synchronising call; the offending access is skipped (loads give 0), so a
+// wrong address is reported, never dereferenced.  Nothing traps or asserts.
+struct DebugRanges {
+  uint64_t lo[3], hi[3];       // state arena, caller's gradient table, exchange buffer (hi exclusive; 0,0 = absent)
+  unsigned long long* status;  // device: [0] violations, [1] first offending address, [2] its kind | bytes << 8
+};                             //         kind 1 = outside every range, 2 = not the row it should be
+#ifdef LA_DEBUG
+#define LA_DBG_ARG(...) , __VA_ARGS__
+__device__ __forceinline__ DebugRanges& dbg_ranges() {
+  __shared__ DebugRanges r;
+  return r;
+}
+__device__ __forceinline__ void dbg_begin(const DebugRanges& from_params) {
+  if (threadIdx.x == 0) dbg_ranges() = from_params;
+  __syncthreads();
+}
+static __device__ __noinline__ void dbg_report(uint64_t addr, unsigned long long kind) {
+  unsigned long long* st = dbg_ranges().status;
+  if (atomicAdd(st, 1ull) == 0ull) {
+    st[1] = addr;
+    st[2] = kind;
+  }
+}
+__device__ __forceinline__ bool dbg_access_ok(const void* ptr, uint32_t bytes) {
+  const DebugRanges& r = dbg_ranges();
+  if (r.status == nullptr) return true;  // unchecked launch (no context behind it)
+  const uint64_t a = reinterpret_cast<uint64_t>(ptr);
+  bool ok = false;
+#pragma unroll
+  for (int k = 0; k < 3; ++k) ok = ok || (a >= r.lo[k] && a + bytes <= r.hi[k]);
+  if (!ok) dbg_report(a, 1ull | ((unsigned long long)bytes << 8));
+  return ok;
+}
+__device__ __forceinline__ void dbg_expect_row(uint64_t addr, uint64_t expected) {
+  if (dbg_ranges().status != nullptr && addr != expected) dbg_report(addr, 2ull);
+}
+#else
+#define LA_DBG_ARG(...)
+#endif
+
 struct SweepParams {
+#ifdef LA_DEBUG
+  DebugRanges dbg;
+#endif
   float* X;        // [W][stride]
   float* B2;       // [W][stride]
   float* Bs;       // [stride]   accumulator as of the last synchronisation
@@ -101,6 +148,13 @@ __device__ __forceinline__ float* as_mut(uint64_t addr) { return reinterpret_cas
 template <int V>
 __device__ __forceinline__ Vec<V> ld_stream(const float* p) {
   Vec<V> r;
+#ifdef LA_DEBUG
+  if (!dbg_access_ok(p, V * sizeof(float))) {
+#pragma unroll
+    for (int k = 0; k < V; ++k) r.v[k] = 0.0f;
+    return r;
+  }
+#endif
   if (V == 4) {
     const float4 t = __ldcs(reinterpret_cast<const float4*>(p));
     r.v[0] = t.x; r.v[1] = t.y; r.v[V - 2] = t.z; r.v[V - 1] = t.w;
@@ -113,6 +167,9 @@ __device__ __forceinline__ Vec<V> ld_stream(const float* p) {
 
 template <int V>
 __device__ __forceinline__ void st_stream(float* p, const Vec<V>& a) {
+#ifdef LA_DEBUG
+  if (!dbg_access_ok(p, V * sizeof(float))) return;
+#endif
   if (V == 4) {
     __stcs(reinterpret_cast<float4*>(p), make_float4(a.v[0], a.v[1], a.v[V - 2], a.v[V - 1]));
   } else {
@@ -316,10 +373,14 @@ struct ReplicaChunk {
 // group and is left pointing at replica i0+CH.  B^2 of a replica sits `b_delta` bytes after x.
 template <int V, int CH, bool ACC = true>
 __device__ __forceinline__ void load_chunk(ReplicaChunk<V, CH>& ch, uint64_t& addr, uint64_t b_delta,
-                                           uint64_t stride_bytes, uint32_t W, uint32_t i0) {
+                                           uint64_t stride_bytes, uint32_t W, uint32_t i0
+                                           LA_DBG_ARG(uint64_t row0_addr)) {  // checked build: address of replica 0
 #pragma unroll
   for (int k = 0; k < CH; ++k)
     if (i0 + k < W) {
+#ifdef LA_DEBUG
+      dbg_expect_row(addr, row0_addr + (uint64_t)(i0 + k) * stride_bytes);
+#endif
       ch.x[k] = ld_stream<V>(as_ptr(addr));
       if (ACC) ch.b[k] = ld_stream<V>(as_ptr(addr + b_delta));
       advance(addr, stride_bytes);
@@ -329,7 +390,11 @@ __device__ __forceinline__ void load_chunk(ReplicaChunk<V, CH>& ch, uint64_t& ad
 // Stores x and B^2 of one replica at `addr` and advances to the next replica.
 template <int V, bool ACC = true>
 __device__ __forceinline__ void store_replica(uint64_t& addr, uint64_t b_delta, uint64_t stride_bytes,
-                                              const Vec<V>& x, const Vec<V>& b) {
+                                              const Vec<V>& x, const Vec<V>& b
+                                              LA_DBG_ARG(uint64_t expected_addr)) {
+#ifdef LA_DEBUG
+  dbg_expect_row(addr, expected_addr);
+#endif
   st_stream<V>(as_mut(addr), x);
   if (ACC) st_stream<V>(as_mut(addr + b_delta), b);
   advance(addr, stride_bytes);
@@ -347,10 +412,19 @@ template <int GM, int V, int CH>
 __device__ __forceinline__ void load_grads(GradChunk<V, CH>& gc, const SweepParams& p, uint64_t& g_addr,
                                            uint64_t row_bytes, uint32_t W, uint32_t i0, uint64_t off) {
   constexpr bool kF32 = (GM == kGradExternalF32);
+  constexpr uint32_t kElem = kF32 ? 4u : 2u;
 #pragma unroll
   for (int k = 0; k < CH; ++k)
     if (i0 + k < W) {
+#ifdef LA_DEBUG
+      dbg_expect_row(g_addr, reinterpret_cast<uint64_t>(p.gext) + (uint64_t)(i0 + k) * row_bytes + off * kElem);
+#endif
       if (p.gext_vec) {
+#ifdef LA_DEBUG
+        if (!dbg_access_ok(reinterpret_cast<const void*>(g_addr), V * kElem)) {
+          gc.g[k] = splat<V>(0.0f);
+        } else
+#endif
         if (kF32) {
           gc.g[k] = ld_stream<V>(as_ptr(g_addr));
         } else {
@@ -371,7 +445,11 @@ __device__ __forceinline__ void load_grads(GradChunk<V, CH>& gc, const SweepPara
 #pragma unroll
         for (int e = 0; e < V; ++e) {
           float v = 0.0f;
-          if (off + e < p.n) {
+          bool take = off + e < p.n;
+#ifdef LA_DEBUG
+          take = take && dbg_access_ok(reinterpret_cast<const void*>(g_addr + e * kElem), kElem);
+#endif
+          if (take) {
             if (kF32) {
               v = __ldcs(reinterpret_cast<const float*>(g_addr) + e);
             } else {
@@ -453,6 +531,9 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
   const uint32_t W = (W_ > 0) ? (uint32_t)W_ : p.W;
   const uint32_t Wr = kImport ? 1u : W;
 
+#ifdef LA_DEBUG
+  dbg_begin(p.dbg);
+#endif
   __shared__ uint64_t keys[kMaxWorkers];
   if (kNeedsNoise) {
     if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, step_index(p), p.identical_workers ? 0u : p.worker_base + threadIdx.x);
@@ -500,7 +581,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
   load_coord<GM, STEP, kLoadsBs, V>(in_next, p, grp * V);
   uint64_t ld_addr = rd_base + grp * (V * sizeof(float));
   uint64_t g_addr = g_base + grp * (V * kGradElem);
-  load_chunk<V, CH, ACC>(nxt, ld_addr, rd_b_delta, stride_bytes, Wr, 0u);
+  load_chunk<V, CH, ACC>(nxt, ld_addr, rd_b_delta, stride_bytes, Wr, 0u LA_DBG_ARG(rd_base + grp * (V * sizeof(float))));
   if (kExternal) load_grads<GM, V, kExternal ? CH : 1>(gnxt, p, g_addr, g_row_bytes, W, 0u, grp * V);
 
   for (;;) {
@@ -521,12 +602,12 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
       ReplicaChunk<V, CH> cur = nxt;
       GradChunk<V, kExternal ? CH : 1> gcur = gnxt;
       if (i0 + CH < Wr) {
-        load_chunk<V, CH, ACC>(nxt, ld_addr, rd_b_delta, stride_bytes, Wr, i0 + CH);
+        load_chunk<V, CH, ACC>(nxt, ld_addr, rd_b_delta, stride_bytes, Wr, i0 + CH LA_DBG_ARG(rd_base + off * sizeof(float)));
         if (kExternal) load_grads<GM, V, kExternal ? CH : 1>(gnxt, p, g_addr, g_row_bytes, W, i0 + CH, off);
       } else if (has_next) {
         load_coord<GM, STEP, kLoadsBs, V>(in_next, p, next_grp * V);
         ld_addr = rd_base + next_grp * (V * sizeof(float));
-        load_chunk<V, CH, ACC>(nxt, ld_addr, rd_b_delta, stride_bytes, Wr, 0u);
+        load_chunk<V, CH, ACC>(nxt, ld_addr, rd_b_delta, stride_bytes, Wr, 0u LA_DBG_ARG(rd_base + next_grp * (V * sizeof(float))));
         if (kExternal) {
           g_addr = g_base + next_grp * (V * kGradElem);
           load_grads<GM, V, kExternal ? CH : 1>(gnxt, p, g_addr, g_row_bytes, W, 0u, next_grp * V);
@@ -546,7 +627,8 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
             if (POST) {
               tree.push_in_chunk(i, k, i0 + CH <= Wr, cur.x[k], cur.b[k]);
             } else {
-              store_replica<V, ACC>(st_addr, b_delta, stride_bytes, cur.x[k], cur.b[k]);
+              store_replica<V, ACC>(st_addr, b_delta, stride_bytes, cur.x[k], cur.b[k]
+                                    LA_DBG_ARG(x_base + off * sizeof(float) + (uint64_t)i * stride_bytes));
             }
           }
         }
@@ -575,11 +657,14 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
             Vec<V> xv = xm, bv = bm;
             const Vec<V> g = gradient<GM, BF16, V>(p, in, xv, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
             apply<V, ACC>(r, g, xv, bv);
-            store_replica<V, ACC>(st_addr, b_delta, stride_bytes, xv, bv);
+            store_replica<V, ACC>(st_addr, b_delta, stride_bytes, xv, bv
+                                  LA_DBG_ARG(x_base + off * sizeof(float) + (uint64_t)i * stride_bytes));
           }
         } else {
 #pragma unroll kWriteUnroll
-          for (uint32_t i = 0; i < W; ++i) store_replica<V, ACC>(st_addr, b_delta, stride_bytes, xm, bm);
+          for (uint32_t i = 0; i < W; ++i)
+            store_replica<V, ACC>(st_addr, b_delta, stride_bytes, xm, bm
+                                  LA_DBG_ARG(x_base + off * sizeof(float) + (uint64_t)i * stride_bytes));
         }
       }
     }
@@ -599,6 +684,9 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_adagrad(const SweepParams p
   constexpr uint64_t kGradElem = (GM == kGradExternalBF16) ? 2 : 4;
   constexpr int kOuterUnroll = (W_ > 0) ? kMaxWorkers : 1;
   const uint32_t W = (W_ > 0) ? (uint32_t)W_ : p.W;
+#ifdef LA_DEBUG
+  dbg_begin(p.dbg);
+#endif
   __shared__ uint64_t keys[kMaxWorkers];
   if (kNeedsNoise) {
     if (threadIdx.x < W) keys[threadIdx.x] = step_worker_key(p.seed, step_index(p), p.identical_workers ? 0u : p.worker_base + threadIdx.x);

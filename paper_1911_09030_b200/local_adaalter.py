@@ -14,9 +14,12 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "liblocal_adaalter.so")
+# LA_LIBRARY=debug selects the checked build (same code compiled with -DLA_DEBUG: every kernel
+# address is range-checked and violations surface as LA_EBOUNDS at the next synchronising call).
+LIB_PATH = os.path.join(_HERE, "liblocal_adaalter_debug.so" if os.environ.get("LA_LIBRARY") == "debug"
+                        else "liblocal_adaalter.so")
 
-LA_OK, LA_EINVAL, LA_ENOMEM, LA_ECUDA, LA_ESTATE, LA_ETOOBIG = 0, -1, -2, -3, -4, -5
+LA_OK, LA_EINVAL, LA_ENOMEM, LA_ECUDA, LA_ESTATE, LA_ETOOBIG, LA_EBOUNDS = 0, -1, -2, -3, -4, -5, -6
 LA_STATIC_SCRATCH_MAX_COORDS = 1048576
 LA_F32, LA_BF16 = 0, 1
 LA_FUSE_NONE, LA_FUSE_STEP_SYNC, LA_FUSE_SYNC_STEP, LA_FUSE_PERIOD = 0, 1, 2, 3
@@ -100,6 +103,8 @@ def lib() -> C.CDLL:
             "la_stream_sync": [vp],
             "la_noise_tables": [vp, vp, vp, vp],
             "la_replica_means_static": [vp, vp, u32, u64, u64, vp, vp, vp],
+            "la_debug_build": [],
+            "la_debug_narrow": [vp, u64],
         }
         for name, args in sig.items():
             fn = getattr(L, name)
@@ -119,6 +124,11 @@ def replica_means_static(x_ptr, b2_ptr, W, n, stride, x_mean_ptr, b2_mean_ptr, s
     return lib().la_replica_means_static(C.c_void_p(int(x_ptr)), C.c_void_p(int(b2_ptr)), int(W), int(n), int(stride),
                                          C.c_void_p(int(x_mean_ptr)), C.c_void_p(int(b2_mean_ptr)),
                                          C.c_void_p(int(stream)) if stream else None)
+
+
+def debug_build() -> bool:
+    """True when the loaded library is the checked build."""
+    return bool(lib().la_debug_build())
 
 
 def noise_tables(radius_ptr=None, cos_ptr=None, sin_ptr=None, stream=None) -> int:
@@ -331,6 +341,10 @@ class LocalAdaAlter:
         f, d = C.c_double(), C.c_double()
         self._ck(self.L.la_diagnostics(self.h, C.byref(f), C.byref(d)))
         return f.value, d.value
+
+    def debug_narrow(self, nbytes):
+        """Checked build only: treat the last `nbytes` bytes of the arena as foreign (0 restores)."""
+        self._ck(self.L.la_debug_narrow(self.h, int(nbytes)))
 
     def sync_stream(self):
         """Block until the context's stream is idle."""

@@ -17,6 +17,7 @@ The engine is anything with the methods used below; the CUDA engine is `CudaEngi
 """
 from __future__ import annotations
 
+import time
 from typing import Optional
 
 
@@ -30,6 +31,7 @@ class WorkerShardedJob:
         self.engine, self.H, self.exchange, self.dist, self.group = engine, int(H), exchange, dist, group
         self.fused = bool(fused) and self.H > 1
         self.syncs = 0
+        self.exchange_seconds = 0.0   # host time between "this rank's sums are ready" and "totals are back"
 
     def _barrier(self):
         if self.dist is not None and self.dist.is_initialized() and self.dist.get_world_size(self.group) > 1:
@@ -43,23 +45,27 @@ class WorkerShardedJob:
 
     def _exchange(self):
         e = self.engine
+        multi = self.dist is not None and self.dist.is_initialized() and self.dist.get_world_size(self.group) > 1
         if self.exchange == "peer":
             e.stream_sync()
+            t0 = time.perf_counter()
             self._barrier()            # every rank's sums are in its buffer
             e.combine()
             e.stream_sync()
             self._barrier()            # every slice of every buffer holds the total
-        else:
+            self.exchange_seconds += time.perf_counter() - t0
+        elif multi:
             buf = e.buffer_tensor()
-            if self.dist is not None and self.dist.is_initialized() and self.dist.get_world_size(self.group) > 1:
-                # The export kernel ran on the context's stream, the collective runs on the process
-                # group's: finish the first before the second reads the buffer, and finish the second
-                # before the import kernel (context stream again) reads the totals.
-                e.stream_sync()
-                self.dist.all_reduce(buf, op=self.dist.ReduceOp.SUM, group=self.group)
-                done = getattr(e, "collective_done", None)
-                if done is not None:
-                    done()
+            # The export kernel ran on the context's stream, the collective runs on the process
+            # group's: finish the first before the second reads the buffer, and finish the second
+            # before the import kernel (context stream again) reads the totals.
+            e.stream_sync()
+            t0 = time.perf_counter()
+            self.dist.all_reduce(buf, op=self.dist.ReduceOp.SUM, group=self.group)
+            done = getattr(e, "collective_done", None)
+            if done is not None:
+                done()
+            self.exchange_seconds += time.perf_counter() - t0
 
     def run(self, T: int):
         """T iterations of Algorithm 3: local step; if t' == H: synchronise."""

@@ -126,42 +126,81 @@ import numpy as np, torch, torch.distributed as dist
 from paper_1911_09030_b200 import local_adaalter as la
 from paper_1911_09030_b200.worker_sharded import CudaEngine, WorkerShardedJob
 from oracle.oracle import Oracle
-dist.init_process_group("gloo")
+mode = os.environ["LA_MODE"]
+dist.init_process_group("gloo")               # host barriers, handle exchange; in the all-reduce mode also the collective
 rank, world = dist.get_rank(), dist.get_world_size()
 torch.cuda.set_device(0)                      # both ranks share the one GPU; no kernel waits for the other rank
-n, W_local, H, T = 40000, 4, 3, 8
+n, W_local, H, T = 40000, 4, 3, 11
 rng = np.random.default_rng(0)
 a = rng.uniform(0.1, 10, n).astype(np.float32); c = rng.standard_normal(n).astype(np.float32)
-g = la.LocalAdaAlter([n], W_local, 0.1, 1.0, la.LA_H_NEVER)
-g.set_grad_quadratic(9, a, c, 0.3)
-eng = CudaEngine(g, rank, world)
-eng.attach_peers(dist)                        # CUDA IPC handles through the process group
-job = WorkerShardedJob(eng, H, exchange="peer", dist=dist)
-job.run(T)
+o = Oracle(n, W_local * world, 0.1, 1.0, H)
+own = torch.cuda.Stream() if mode == "allreduce_fused_own_stream" else None
+g = la.LocalAdaAlter([n], W_local, 0.1, 1.0, la.LA_H_NEVER, stream=own.cuda_stream if own else None)
+if mode == "supplied":
+    # caller-supplied gradients: every rank draws the full [W_total][n] table from the same seed and
+    # passes its own rows; the step that completes a period is fused with the export
+    eng = CudaEngine(g, rank, world)
+    eng.attach_peers(dist)
+    job = WorkerShardedJob(eng, H, exchange="peer", dist=dist)
+    grng = np.random.default_rng(1)
+    for t in range(1, T + 1):
+        G = grng.standard_normal((W_local * world, n)).astype(np.float32)
+        if rank == 0:
+            o.local_step(G)
+        Gd = torch.from_numpy(G[rank * W_local:(rank + 1) * W_local].copy()).cuda()
+        if t % H == 0:
+            g.comm_step_grads_export(Gd.data_ptr(), la.LA_F32)
+            job._exchange()
+            g.comm_import()
+            if rank == 0:
+                o.sync()
+        else:
+            g.local_step_grads(Gd.data_ptr(), la.LA_F32)
+        g.stream_sync()                       # Gd is released at the end of the iteration
+else:
+    g.set_grad_quadratic(9, a, c, 0.3)
+    o.set_grad_quadratic(9, a, c, 0.3)
+    eng = CudaEngine(g, rank, world)
+    eng.attach_peers(dist)                    # CUDA IPC handles through the process group
+    job = WorkerShardedJob(eng, H, exchange="allreduce" if mode.startswith("allreduce") else "peer", dist=dist,
+                           fused=mode != "peer")
+    job.run(5)                                # ends inside a period ...
+    job.run(T - 5)                            # ... and the schedule carries on
+    assert job.syncs == T // H
+    if rank == 0:
+        o.run(T)
 g.stream_sync()
 mine = [g.read_state(i) for i in range(W_local)]
 parts = [None] * world
-dist.all_gather_object(parts, (rank, mine, g.get_counters()))
+dist.all_gather_object(parts, (rank, mine, g.get_counters(), g.get_stats()))
 dist.barrier()
 if rank == 0:
-    o = Oracle(n, W_local * world, 0.1, 1.0, H)
-    o.set_grad_quadratic(9, a, c, 0.3)
-    o.run(T)
-    for r, st, cnt in parts:
-        assert cnt == o.counters()
+    for r, st, cnt, stats in parts:
+        assert cnt == o.counters(), (cnt, o.counters())
+        if mode != "peer":
+            assert stats["launches_fused"] >= T // H          # the exchange-fused kernels ran
         for i in range(W_local):
             for u, v in zip(st[i], o.read(r * W_local + i)):
                 assert np.array_equal(u.view(np.uint32), v.view(np.uint32)), (r, i)
-    print("IPC_PEER_OK")
+    print("IPC_PEER_OK", mode)
 g.close()
 dist.destroy_process_group()
 '''
 
 
-def test_two_processes_exchange_through_cuda_ipc(tmp_path):
+@pytest.mark.parametrize("mode", ["peer", "peer_fused", "allreduce_fused_own_stream", "supplied"])
+def test_two_processes_exchange_through_cuda_ipc(tmp_path, mode):
     """Two OS processes (gloo for the host-side barriers and the handle exchange) map each other's
-    exchange buffer with CUDA IPC and synchronise with the peer-load combine kernel; the result is
-    the oracle's with W_total workers, bitwise.  Both processes use the same GPU here."""
+    exchange buffer with CUDA IPC and synchronise across the process boundary; the result is the
+    oracle's with W_total workers, bitwise.  Both processes use the same GPU here.
+      peer                        export, peer-load combine kernel, import
+      peer_fused                  the steps next to a synchronisation fused with the exchange
+                                  (step+export, combine, import+step)
+      allreduce_fused_own_stream  the same with the buffer all-reduced by torch.distributed (two ranks:
+                                  one addition per element, so still bitwise) and the context on a
+                                  stream of its own, so the ordering between the context's stream
+                                  and the collective is what makes it pass
+      supplied                    caller-supplied gradient tables, the closing step fused with the export"""
     import os, socket, subprocess, sys
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     script = tmp_path / "ipc_worker.py"
@@ -169,12 +208,12 @@ def test_two_processes_exchange_through_cuda_ipc(tmp_path):
     with socket.socket() as s:
         s.bind(("127.0.0.1", 0))
         port = s.getsockname()[1]
-    env = dict(os.environ, LA_ROOT=root, MASTER_ADDR="127.0.0.1")
+    env = dict(os.environ, LA_ROOT=root, MASTER_ADDR="127.0.0.1", LA_MODE=mode)
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
            "--master-addr", "127.0.0.1", "--master-port", str(port), str(script)]
     r = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=300)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-4000:]
-    assert "IPC_PEER_OK" in r.stdout
+    assert "IPC_PEER_OK " + mode in r.stdout
 
 
 @pytest.mark.parametrize("H,T", [(2, 9), (3, 10), (4, 8), (5, 5), (1, 4)])
