@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(LA_BLOCK) la_combine_sums(const CombineParams 
       const Vec<V> sb = ld_stream<V>(p.S[r] + p.stride + off);
       tree.push(r, sx, sb);
     }
-    tree.finish();
+    tree.finish(p.world);
     for (uint32_t r = 0; r < p.world; ++r) {
       st_stream<V>(p.S[r] + off, tree.x[0]);
       st_stream<V>(p.S[r] + p.stride + off, tree.b[0]);

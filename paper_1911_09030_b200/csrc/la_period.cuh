@@ -122,7 +122,7 @@ __global__ void __launch_bounds__(LA_PERIOD_BLOCK, MINB) la_period(const PeriodP
         }
     }
     if (POST) {
-      tree.finish();
+      tree.finish(W);
       const Vec<V> xm = div_by_workers<W_, V>(tree.x[0], W);
       const Vec<V> bm = div_by_workers<W_, V>(tree.b[0], W);
       st_stream<V>(p.Bs + off, bm);

@@ -126,6 +126,9 @@ constexpr int kTreeDepth = 7;  // log2(kMaxWorkers) + 1 partial sums
 #ifndef LA_CH
 #define LA_CH 4
 #endif
+#ifndef LA_CH_V4
+#define LA_CH_V4 2
+#endif
 constexpr int kBlockThreads = LA_BLOCK;
 
 // V consecutive coordinates held by one thread (V = 4: one 128-bit access, two Box-Muller
@@ -220,27 +223,34 @@ __device__ __forceinline__ Vec<V> div_by_workers(const Vec<V>& a, uint32_t W) {
 template <int V, bool ACC = true>
 struct PairTree {
   Vec<V> x[kTreeDepth], b[ACC ? kTreeDepth : 1];
-  int sp = 0;
+  // Before worker i is pushed the stack holds one entry per set bit of i, so every position
+  // follows from i alone (no running stack pointer to carry through the unrolled code): the new
+  // entry goes to slot popcount(i) and is merged downwards once per trailing one bit of i.
   __device__ __forceinline__ void push(uint32_t i, const Vec<V>& vx, const Vec<V>& vb) {
-    x[sp] = vx;
-    if (ACC) b[ACC ? sp : 0] = vb;
-    ++sp;
-    for (uint32_t cnt = i + 1u; (cnt & 1u) == 0u; cnt >>= 1) {
-      --sp;
-      x[sp - 1] = add(x[sp - 1], x[sp]);
-      if (ACC) b[ACC ? sp - 1 : 0] = add(b[ACC ? sp - 1 : 0], b[ACC ? sp : 0]);
-    }
+    const int top = __popc(i);
+    const int merges = __popc(i & ~(i + 1u));
+    x[top] = vx;
+    if (ACC) b[ACC ? top : 0] = vb;
+#pragma unroll
+    for (int m = 0; m < kTreeDepth - 1; ++m)
+      if (m < merges) {
+        x[top - 1 - m] = add(x[top - 1 - m], x[top - m]);
+        if (ACC) b[ACC ? top - 1 - m : 0] = add(b[ACC ? top - 1 - m : 0], b[ACC ? top - m : 0]);
+      }
   }
   // position k within a chunk of replicas is irrelevant here (see PairTreeDyn)
   __device__ __forceinline__ void push_in_chunk(uint32_t i, int, bool, const Vec<V>& vx, const Vec<V>& vb) {
     push(i, vx, vb);
   }
-  __device__ __forceinline__ void finish() {
-    while (sp > 1) {
-      --sp;
-      x[sp - 1] = add(x[sp - 1], x[sp]);
-      if (ACC) b[ACC ? sp - 1 : 0] = add(b[ACC ? sp - 1 : 0], b[ACC ? sp : 0]);
-    }
+  // After n pushes: merge what is left, older entries on the left; the total ends in slot 0.
+  __device__ __forceinline__ void finish(uint32_t n) {
+    const int sp = __popc(n);
+#pragma unroll
+    for (int m = 0; m < kTreeDepth - 1; ++m)
+      if (m < sp - 1) {
+        x[sp - 2 - m] = add(x[sp - 2 - m], x[sp - 1 - m]);
+        if (ACC) b[ACC ? sp - 2 - m : 0] = add(b[ACC ? sp - 2 - m : 0], b[ACC ? sp - 1 - m : 0]);
+      }
   }
 };
 
@@ -317,7 +327,7 @@ struct PairTreeDyn {
 
   // Leaves the total in x[0], b[0]: the occupied levels are merged from the lowest up, each
   // higher (older) level on the left.
-  __device__ __forceinline__ void finish() {
+  __device__ __forceinline__ void finish(uint32_t) {
     Vec<V> ax = x[0], ab = b[0];
     bool have = false;
 #pragma unroll
@@ -525,7 +535,9 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
   constexpr bool kExport = (XCH == 1), kImport = (XCH == 2);
   constexpr bool kNeedsNoise = STEP && (GM == kGradNoise || GM == kGradNoiseScaled || GM == kGradQuadratic);
   constexpr int WR_ = kImport ? 1 : W_;  // replicas on the READ side (import: the one row of totals)
-  constexpr int CH = (WR_ > 0) ? (WR_ < LA_CH ? WR_ : LA_CH) : 4;  // replicas loaded before any is consumed
+  // replicas loaded before any is consumed (four-coordinate threads hold twice the data per replica)
+  constexpr int kChunkMax = (V == 4) ? LA_CH_V4 : LA_CH;
+  constexpr int CH = (WR_ > 0) ? (WR_ < kChunkMax ? WR_ : kChunkMax) : 4;
   constexpr int kReadUnroll = (WR_ > 0) ? kMaxWorkers : 1;  // static counts: unroll fully, so that the
   constexpr int kWriteUnroll = (W_ > 0) ? kMaxWorkers : 1;  // reduction stack is indexed by constants
   const uint32_t W = (W_ > 0) ? (uint32_t)W_ : p.W;
@@ -597,8 +609,10 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
     if (!ACC) r = splat<V>(eta_t);
     typename TreeFor<WR_, V, ACC>::type tree;
 
-#pragma unroll kReadUnroll
-    for (uint32_t i0 = 0; i0 < Wr; i0 += CH) {
+    // One chunk of CH replicas starting at replica i0: start the loads of what comes next, then
+    // consume the chunk.  `tr` is the reduction the chunk's results enter, `local0` the index of
+    // the chunk's first replica as that reduction counts it, `whole` whether all CH replicas exist.
+    auto chunk = [&](const uint32_t i0, auto& tr, const uint32_t local0, const bool whole) __attribute__((always_inline)) {
       ReplicaChunk<V, CH> cur = nxt;
       GradChunk<V, kExternal ? CH : 1> gcur = gnxt;
       if (i0 + CH < Wr) {
@@ -616,26 +630,59 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
       asm volatile("" ::: "memory");
 #pragma unroll
       for (int k = 0; k < CH; ++k)
-        if (i0 + k < Wr) {
+        if (whole || i0 + k < Wr) {
           const uint32_t i = i0 + k;
           if (PRE) {
-            tree.push_in_chunk(i, k, i0 + CH <= Wr, cur.x[k], cur.b[k]);
+            tr.push_in_chunk(local0 + k, k, whole, cur.x[k], cur.b[k]);
           } else {
             const Vec<V> g = kExternal ? gcur.g[kExternal ? k : 0]
                                        : gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
             apply<V, ACC>(r, g, cur.x[k], cur.b[k]);
             if (POST) {
-              tree.push_in_chunk(i, k, i0 + CH <= Wr, cur.x[k], cur.b[k]);
+              tr.push_in_chunk(local0 + k, k, whole, cur.x[k], cur.b[k]);
             } else {
               store_replica<V, ACC>(st_addr, b_delta, stride_bytes, cur.x[k], cur.b[k]
                                     LA_DBG_ARG(x_base + off * sizeof(float) + (uint64_t)i * stride_bytes));
             }
           }
         }
+    };
+
+    if constexpr (WR_ > 0) {
+#pragma unroll kReadUnroll
+      for (uint32_t i0 = 0; i0 < Wr; i0 += CH) chunk(i0, tree, i0, i0 + CH <= Wr);
+    } else {
+      // Worker count known only at run time.  Passes that average first take whole tiles of
+      // kTile replicas: inside a tile every position is a compile-time constant, so the tile is
+      // summed by the stack-form tree (constant register indices, no predication) and enters the
+      // run-time counter as one aligned block — an aligned block of 2^k workers is a complete
+      // subtree of the adjacent-pair tree.  What is left (fewer than kTile replicas) goes through
+      // the counter chunk by chunk.
+      constexpr int kTile = 16, kTileLog = 4;
+      static_assert(kTile % CH == 0 && (kTile / 2) % CH == 0, "tiles are whole chunks");
+      uint32_t i0 = 0;
+      if ((PRE || POST) && V == 2) {  // (four-coordinate threads have no registers to spare for a tile)
+        for (; i0 + kTile <= Wr; i0 += kTile) {
+          PairTree<V, ACC> tile;
+#pragma unroll
+          for (int c = 0; c < kTile / CH; ++c) chunk(i0 + c * CH, tile, c * CH, true);
+          tile.finish(kTile);
+          tree.template push_block<kTileLog>(tile.x[0], tile.b[0]);
+        }
+        if (i0 + kTile / 2 <= Wr) {  // one half tile, the same way
+          PairTree<V, ACC> tile;
+#pragma unroll
+          for (int c = 0; c < kTile / 2 / CH; ++c) chunk(i0 + c * CH, tile, c * CH, true);
+          tile.finish(kTile / 2);
+          tree.template push_block<kTileLog - 1>(tile.x[0], tile.b[0]);
+          i0 += kTile / 2;
+        }
+      }
+      for (; i0 < Wr; i0 += CH) chunk(i0, tree, i0, i0 + CH <= Wr);
     }
 
     if (PRE || POST) {
-      tree.finish();
+      tree.finish(Wr);
       if (kExport) {
         // the means are formed after the exchange, from the totals over all ranks
         st_stream<V>(p.xch + off, tree.x[0]);
@@ -721,7 +768,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_adagrad(const SweepParams p
       }
       tree.push(i, g, g);
     }
-    tree.finish();
+    tree.finish(W);
     const Vec<V> gm = div_by_workers<W_, V>(tree.x[0], W);
 #pragma unroll
     for (int k = 0; k < V; ++k) {
