@@ -698,14 +698,13 @@ def run_report(args):
 def run_kernel_report(args):
     """Per-kernel GB/s away from the benchmark configurations: worker counts with their own
     instantiation (3, 6, 12), worker counts known only at run time (5, 24, 32, 64), and
-    caller-supplied gradient tables in fp32 and bf16 (W = 4, 8, 16).  N = 2^24, pure-noise gradients
+    caller-supplied gradient tables in fp32 and bf16 (W = 4, 8, 16).  N = 2^24 (more for W < 4), pure-noise gradients
     (the shape of configuration 4), every pass timed by CUDA events around the launch.
     Markdown table to stdout, JSON to --report-out."""
     import torch
     from paper_1911_09030_b200 import local_adaalter as la
     torch.cuda.set_device(0)
     peak, peak_kind = measured_peak()
-    N = args.N or (1 << 24)
     rows = []
 
     def classes(ctx, W, what):
@@ -715,12 +714,16 @@ def run_kernel_report(args):
             if n and st[f"ms_{cls}"] > 0:
                 ms = st[f"ms_{cls}"] / n
                 gbs = st[f"bytes_{cls}"] / n / (ms * 1e-3) / 1e9
-                rows.append({"W": W, "gradients": what, "kernel": KERNEL_NAMES[cls], "launches": int(n),
+                rows.append({"W": W, "N": ctx.N, "gradients": what, "kernel": KERNEL_NAMES[cls], "launches": int(n),
                              "us_per_launch": 1e3 * ms, "GBps": gbs, "frac": gbs / peak})
 
     for W in args.workers:
+        # at least 2^26 worker*params per pass, so that a launch lasts long enough to be bandwidth-bound
+        N = args.N or max(1 << 24, 1 << (26 - max(0, W.bit_length() - 1)))
         ctx = la.LocalAdaAlter.with_torch_arena([N], W, 0.01, 1e-2, 4)
         ctx.set_grad_noise(4, None)
+        if args.blocks_per_sm:
+            ctx.set_launch_shape(args.blocks_per_sm)
         for fusion in (la.LA_FUSE_NONE, la.LA_FUSE_STEP_SYNC, la.LA_FUSE_SYNC_STEP):
             ctx.set_fusion(fusion)
             ctx.run(8)
@@ -748,15 +751,15 @@ def run_kernel_report(args):
                 del G
         ctx.close()
         torch.cuda.empty_cache()
-    doc = {"N": N, "peak_GBps": peak, "peak_kind": peak_kind, "rows": rows}
+    doc = {"peak_GBps": peak, "peak_kind": peak_kind, "rows": rows}
     if args.report_out:
         os.makedirs(os.path.dirname(os.path.abspath(args.report_out)), exist_ok=True)
         with open(args.report_out, "w") as f:
             json.dump(doc, f, indent=1)
-    print(f"| W | gradients | kernel | launches | us per launch | GB/s | of {peak:.0f} ({peak_kind}) |")
-    print("|---|---|---|---|---|---|---|")
+    print(f"| W | N | gradients | kernel | launches | us per launch | GB/s | of {peak:.0f} ({peak_kind}) |")
+    print("|---|---|---|---|---|---|---|---|")
     for r in rows:
-        print(f"| {r['W']} | {r['gradients']} | {r['kernel']} | {r['launches']} | {r['us_per_launch']:.1f} | "
+        print(f"| {r['W']} | {r['N']} | {r['gradients']} | {r['kernel']} | {r['launches']} | {r['us_per_launch']:.1f} | "
               f"{r['GBps']:.0f} | {r['frac']:.3f} |")
 
 
@@ -820,7 +823,8 @@ def main():
     ap.add_argument("--H", type=int, default=None, help="override the synchronisation period")
     ap.add_argument("--T", type=int, default=None, help="override iterations per step")
     ap.add_argument("--N", type=int, default=None, help="override the size (one flat tensor), e.g. for small ncu captures")
-    ap.add_argument("--fusion", type=int, default=1, help="0 unfused, 1 step+sync, 2 sync+next step")
+    ap.add_argument("--fusion", type=int, default=1,
+                    help="0 unfused, 1 step+sync, 2 sync+next step, 3 temporal blocking, 4 synchronised state stored once")
     ap.add_argument("--blocks-per-sm", type=int, default=0)
     ap.add_argument("--sharding", default="coordinate", choices=["coordinate", "worker"],
                     help="coordinate: every rank owns a coordinate range, no collective (the headline); "

@@ -51,9 +51,18 @@ enum {
 enum { LA_F32 = 0, LA_BF16 = 1 };               /* gradient dtype */
 enum { LA_FUSE_NONE = 0, LA_FUSE_STEP_SYNC = 1, /* la_run: step t'=H and its sync in one pass */
        LA_FUSE_SYNC_STEP = 2,                   /* la_run: sync folded into the following step */
-       LA_FUSE_PERIOD = 3 };                    /* la_run: up to 8 consecutive local steps (and the sync
+       LA_FUSE_PERIOD = 3,                      /* la_run: up to 8 consecutive local steps (and the sync
                                                    that closes the period) in one pass over HBM; for the
                                                    generated gradients, whose noise lives in registers */
+       LA_FUSE_MEAN_ONCE = 4 };                 /* la_run: a synchronisation makes all replicas equal, so its
+                                                   result is stored once: the step t'=H writes only the sums of
+                                                   its y, A^2 over the workers (into replica 0's rows) and the
+                                                   step t'=1 that follows reads that one copy; per period one
+                                                   write and one read of W-1 replicas fewer than LA_FUSE_STEP_SYNC.
+                                                   Generated gradients, Local AdaAlter, H >= 2 (otherwise it
+                                                   behaves as LA_FUSE_STEP_SYNC).  Between the two steps, also
+                                                   across calls, the means are pending; every call that looks
+                                                   at or changes the state completes them first. */
 enum { LA_RULE_ADAALTER = 0,  /* Algorithm 3, Local AdaAlter (default) */
        LA_RULE_LOCAL_SGD = 1, /* Algorithm 2: y = x - eta G, x averaged every H steps, no accumulator */
        LA_RULE_ADAGRAD = 2 }; /* Algorithm 1: gradients averaged every step, B^2 += G o G, updated B^2 divides */
@@ -137,8 +146,8 @@ int la_set_rule(la_ctx* ctx, int rule);
 int la_set_fusion(la_ctx* ctx, int mode);
 /* Tuning knob: the sweep kernels run as a grid-stride loop over at most
  * blocks_per_sm * (number of SMs) blocks of 256 threads; 0 restores the built-in
- * per-kernel defaults (96 for kernels that take a step, 768 for the temporal-blocking
- * kernel, unbounded for the pure sync). */
+ * per-kernel defaults (16 per replica up to 96 for kernels that take a step, 768 for the
+ * temporal-blocking kernel, unbounded for the pure sync). */
 int la_set_launch_shape(la_ctx* ctx, int blocks_per_sm);
 /* Launch-bound regime (small N, e.g. a 2 MB state where a step takes a few microseconds): let
  * la_run replay whole periods of H iterations from a captured CUDA graph instead of launching

@@ -195,6 +195,9 @@ struct la_ctx {
   int fusion = LA_FUSE_NONE;
   int rule = LA_RULE_ADAALTER;
   bool shared_iterate = false;  // AdaGrad steps ran: replica 0 holds x_t, B^2_t; replicas 1..W-1 are stale
+  bool sums_in_replica0 = false;  // LA_FUSE_MEAN_ONCE between a closing step and the next one: replica 0's rows hold
+                                  // the tree SUMS of that step's y, A^2; the other replicas and the stale array are
+                                  // out of date until the sums are imported (by the next step, or on demand)
   bool profiling = false;
   int device = 0;
   cudaStream_t stream = nullptr;
@@ -397,8 +400,9 @@ double pass_bytes(const la_ctx* c, bool pre, bool step, bool post, int gm) {
 
 // xch: 0 = a pass of the single-GPU path; 1 / 2 = the pass exports to / imports from the exchange
 // buffer of the by-worker sharding (see la_exchange.cuh).
+// in_replica0: the sums live in replica 0's own rows (single-GPU LA_FUSE_MEAN_ONCE) instead of the exchange buffer.
 int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t tp, int gm, const void* gext,
-                 int xch = 0) {
+                 int xch = 0, bool in_replica0 = false) {
   const la::SweepKernel k =
       la::lookup_sweep((int)c->W, c->rule, gm, c->bf16 && gm <= la::kGradQuadratic, pre, step, post, xch);
   la::SweepFn fn = k.fn;
@@ -420,22 +424,27 @@ int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t
   p.warm_up_steps = c->warm_up_steps; p.identical_workers = c->identical ? 1u : 0u;
   p.worker_base = c->worker_base;
   p.eta = c->eta; p.eps = c->eps; p.sigma = c->sigma;
-  p.xch = c->S; p.W_total = c->W_total;
+  p.xch = c->S; p.xch_b_off = c->stride; p.W_total = c->W_total;
+  if (in_replica0) { p.xch = c->X; p.xch_b_off = (uint64_t)c->W * c->stride; p.W_total = c->W; }
 #ifdef LA_DEBUG
   fill_debug_ranges(c, &p.dbg, gext, gext ? (uint64_t)c->W * c->N * (gm == la::kGradExternalBF16 ? 2u : 4u) : 0u);
 #endif
   const unsigned block = la::kBlockThreads;
   const uint64_t ngroups = (c->N + (uint64_t)k.vec - 1) / (uint64_t)k.vec;
   uint64_t blocks = (ngroups + block - 1) / block;
-  // Measured on B200 (sweep of 6..4096 blocks per SM): kernels that take a step run best when a
-  // thread handles a few coordinate groups (96 blocks per SM in the grid: the software pipeline
-  // pays off while blocks stay small enough to balance the SMs); the pure averaging kernel runs
-  // best with one group per thread.
-  const int bps = c->blocks_per_sm > 0 ? c->blocks_per_sm : (step ? 96 : 4096);
+  // Measured on B200 (sweeps of 4..4096 blocks per SM): kernels that take a step run best when a
+  // block lives long enough to amortise its start (the software pipeline over coordinate groups
+  // pays off) yet stays small enough to balance the SMs.  The work of a block grows with the
+  // replicas and coordinates a thread owns, so the grid does too: 16 W blocks per SM for
+  // two-coordinate threads (W = 4: 64; 96 from W = 6 on), half of that for four-coordinate
+  // threads.  The pure averaging kernel runs best with one group per thread.
+  int step_bps = 16 * (int)c->W * 2 / k.vec;
+  step_bps = step_bps < 8 ? 8 : (step_bps > 96 ? 96 : step_bps);
+  const int bps = c->blocks_per_sm > 0 ? c->blocks_per_sm : (step ? step_bps : 4096);
   const uint64_t cap = (uint64_t)c->num_sms * (uint64_t)bps;
   if (blocks > cap) blocks = cap;
   int cls = !step ? kClassSync : (post ? kClassStepSync : (pre ? kClassSyncStep : kClassLocal));
-  if (xch != 0) cls = step ? kClassFused : kClassOther;  // exchange passes: aggregate classes only
+  if (xch != 0 && !in_replica0) cls = step ? kClassFused : kClassOther;  // exchange passes: aggregate classes only
   EventPair ep{};
   if (c->profiling) {
     int rc = begin_timed(c, cls, &ep);
@@ -543,6 +552,17 @@ int materialise_replicas(la_ctx* c) {
     c->stats.launches_other++;
   }
   c->shared_iterate = false;
+  return LA_OK;
+}
+
+// LA_FUSE_MEAN_ONCE leaves the sums of a closing step in replica 0's rows; whoever needs the
+// synchronised state itself (a reader, a writer, another kind of step) first turns them into
+// the means in every replica and the stale array: the import half of that synchronisation.
+int import_pending_sums(la_ctx* c) {
+  if (!c->sums_in_replica0) return LA_OK;
+  int rc = launch_sweep(c, true, false, false, c->t, 0, la::kGradNoise, nullptr, 2, true);
+  if (rc) return rc;
+  c->sums_in_replica0 = false;
   return LA_OK;
 }
 
@@ -675,6 +695,7 @@ int la_set_init(la_ctx* c, const float* x0_host, float b0sq) {
   int rc = do_fill(c, x0_dev);
   if (rc) return rc;
   c->shared_iterate = false;
+  c->sums_in_replica0 = false;
   c->t = 0; c->tp = 0; c->nsync = 0;
   return LA_OK;
 }
@@ -730,7 +751,8 @@ int la_set_warmup(la_ctx* c, uint32_t steps) {
 
 int la_set_fusion(la_ctx* c, int mode) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
-  if (mode != LA_FUSE_NONE && mode != LA_FUSE_STEP_SYNC && mode != LA_FUSE_SYNC_STEP && mode != LA_FUSE_PERIOD)
+  if (mode != LA_FUSE_NONE && mode != LA_FUSE_STEP_SYNC && mode != LA_FUSE_SYNC_STEP && mode != LA_FUSE_PERIOD &&
+      mode != LA_FUSE_MEAN_ONCE)
     return fail(c, LA_EINVAL, "unknown fusion mode %d", mode);
   c->fusion = mode;
   return LA_OK;
@@ -741,6 +763,11 @@ int la_set_rule(la_ctx* c, int rule) {
   if (rule != LA_RULE_ADAALTER && rule != LA_RULE_LOCAL_SGD && rule != LA_RULE_ADAGRAD)
     return fail(c, LA_EINVAL, "unknown update rule %d", rule);
   if (c->tp != 0) return fail(c, LA_ESTATE, "the update rule can only change right after a synchronisation (t' = 0)");
+  if (rule != c->rule) {
+    DeviceGuard guard(c->device);
+    int rc = import_pending_sums(c);
+    if (rc) return rc;
+  }
   if (c->rule == LA_RULE_ADAGRAD && rule != LA_RULE_ADAGRAD) {
     DeviceGuard guard(c->device);
     int rc = materialise_replicas(c);  // the other rules advance every replica on its own
@@ -781,6 +808,7 @@ int la_set_launch_shape(la_ctx* c, int blocks_per_sm) {
 int la_local_step(la_ctx* c) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   DeviceGuard guard(c->device);
+  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
   int rc = launch_sweep(c, false, true, false, c->t + 1, c->tp + 1, c->grad_kind, nullptr);
   if (rc) return rc;
   c->t += 1;
@@ -794,6 +822,7 @@ int la_local_step_grads(la_ctx* c, const void* g_dev, int dtype) {
   if (!g_dev) return fail(c, LA_EINVAL, "g_dev is NULL");
   if (dtype != LA_F32 && dtype != LA_BF16) return fail(c, LA_EINVAL, "dtype must be LA_F32 or LA_BF16");
   DeviceGuard guard(c->device);
+  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
   int rc = launch_sweep(c, false, true, false, c->t + 1, c->tp + 1,
                         dtype == LA_F32 ? la::kGradExternalF32 : la::kGradExternalBF16, g_dev);
   if (rc) return rc;
@@ -809,6 +838,7 @@ int la_step_grads(la_ctx* c, const void* g_dev, int dtype) {
   if (dtype != LA_F32 && dtype != LA_BF16) return fail(c, LA_EINVAL, "dtype must be LA_F32 or LA_BF16");
   if (c->rule == LA_RULE_ADAGRAD) return la_local_step_grads(c, g_dev, dtype);  // Algorithm 1: one pass is the whole iteration
   DeviceGuard guard(c->device);
+  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
   const int gm = dtype == LA_F32 ? la::kGradExternalF32 : la::kGradExternalBF16;
   const bool closes = (c->tp + 1 == c->H);
   if (closes && c->fusion != LA_FUSE_NONE) {
@@ -828,6 +858,7 @@ int la_sync(la_ctx* c) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   if (c->rule == LA_RULE_ADAGRAD) return fail(c, LA_ESTATE, "Distributed AdaGrad keeps one shared iterate: nothing to synchronise");
   DeviceGuard guard(c->device);
+  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
   int rc = launch_sweep(c, true, false, false, c->t, 0, la::kGradNoise, nullptr);
   if (rc) return rc;
   c->tp = 0; c->nsync += 1;
@@ -890,7 +921,8 @@ int la_run(la_ctx* c, uint64_t T) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   DeviceGuard guard(c->device);
   // Launch-bound regime (small N): replay whole periods from a captured graph.
-  if (c->use_graph && !c->profiling && c->rule != LA_RULE_ADAGRAD && c->fusion != LA_FUSE_SYNC_STEP && c->tp == 0 &&
+  if (c->use_graph && !c->profiling && c->rule != LA_RULE_ADAGRAD && c->fusion != LA_FUSE_SYNC_STEP &&
+      c->fusion != LA_FUSE_MEAN_ONCE && !c->sums_in_replica0 && c->tp == 0 &&
       c->H <= 4096u && T >= (uint64_t)c->H) {
     int rc = ensure_period_graph(c);
     if (rc) return rc;
@@ -919,6 +951,10 @@ int la_run(la_ctx* c, uint64_t T) {
 static int run_steps(la_ctx* c, uint64_t T) {
   // Algorithm 3: for t in [T]: local step; if mod(t, H) == 0 (tracked as t' == H): synchronise.
   // `deferred` marks a synchronisation that is due but has been folded into the next step.
+  if (c->fusion != LA_FUSE_MEAN_ONCE || c->rule != LA_RULE_ADAALTER || c->H < 2u) {
+    int rc_ = import_pending_sums(c);
+    if (rc_) return rc_;
+  }
   if (c->rule == LA_RULE_ADAGRAD) {  // Algorithm 1: every iteration is one fully synchronous pass
     for (uint64_t k = 0; k < T; ++k) {
       int rc = la_local_step(c);
@@ -950,8 +986,35 @@ static int run_steps(la_ctx* c, uint64_t T) {
     }
     return LA_OK;
   }
+  if (c->fusion == LA_FUSE_MEAN_ONCE && c->rule == LA_RULE_ADAALTER && c->H >= 2u) {
+    // A synchronisation makes all replicas equal, so its result is stored ONCE: the step that
+    // closes a period writes only the tree sums of its y, A^2 (into replica 0's rows), and the
+    // first step of the next period reads that one copy, divides, and writes the W replicas it
+    // produces.  Per period this saves one write and one read of all replicas but one.  The
+    // sums stay pending across calls; anything else that needs the state imports them first.
+    for (uint64_t k = 0; k < T; ++k) {
+      int rc;
+      if (c->sums_in_replica0) {
+        rc = launch_sweep(c, true, true, false, c->t + 1, 1u, c->grad_kind, nullptr, 2, true);  // import, then step t' = 1
+        if (rc) return rc;
+        c->sums_in_replica0 = false;
+        c->t += 1; c->tp = 1;
+      } else if (c->tp + 1 == c->H) {
+        rc = launch_sweep(c, false, true, true, c->t + 1, c->tp + 1, c->grad_kind, nullptr, 1, true);  // step t' = H, sums only
+        if (rc) return rc;
+        c->sums_in_replica0 = true;
+        c->t += 1; c->tp = 0; c->nsync += 1;
+      } else {
+        rc = la_local_step(c);  // K1
+        if (rc) return rc;
+      }
+    }
+    return LA_OK;
+  }
+  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
   bool deferred = false;
-  const int fusion = (c->fusion == LA_FUSE_PERIOD) ? LA_FUSE_STEP_SYNC : c->fusion;  // baselines: step+sync
+  const int fusion = (c->fusion == LA_FUSE_PERIOD || c->fusion == LA_FUSE_MEAN_ONCE) ? LA_FUSE_STEP_SYNC
+                                                                                      : c->fusion;  // fall-backs: step+sync
   for (uint64_t k = 0; k < T; ++k) {
     int rc;
     if (deferred) {
@@ -986,6 +1049,7 @@ int la_read_range(la_ctx* c, uint32_t worker, uint64_t j0, uint64_t n, float* x_
   if (worker >= c->W) return fail(c, LA_EINVAL, "worker %u out of range (W=%u)", worker, c->W);
   if (j0 > c->N || n > c->N - j0) return fail(c, LA_EINVAL, "coordinate range out of bounds");
   DeviceGuard guard(c->device);
+  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
   if (c->shared_iterate) worker = 0;  // Algorithm 1: every worker holds the one iterate, stored in replica 0
   const size_t bytes = n * sizeof(float);
   if (n) {
@@ -1006,6 +1070,7 @@ int la_write_state(la_ctx* c, uint32_t worker, const float* x_host, const float*
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   if (worker >= c->W) return fail(c, LA_EINVAL, "worker %u out of range (W=%u)", worker, c->W);
   DeviceGuard guard(c->device);
+  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
   if (x_host || b2_host) {
     int rc = materialise_replicas(c);  // a per-worker write: the replicas become individual again
     if (rc) return rc;
@@ -1128,6 +1193,7 @@ int la_comm_export(la_ctx* c) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
   DeviceGuard guard(c->device);
+  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
   return launch_sweep(c, true, false, false, c->t, 0, la::kGradNoise, nullptr, 1);
 }
 
@@ -1160,6 +1226,7 @@ int la_comm_import(la_ctx* c) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
   DeviceGuard guard(c->device);
+  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
   int rc = launch_sweep(c, true, false, false, c->t, 0, la::kGradNoise, nullptr, 2);
   if (rc) return rc;
   c->tp = 0; c->nsync += 1;
@@ -1170,6 +1237,7 @@ static int step_export_impl(la_ctx* c, int gm, const void* gext) {
   if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
   if (c->rule != LA_RULE_ADAALTER) return fail(c, LA_ESTATE, "sharding by worker is implemented for Local AdaAlter only");
   DeviceGuard guard(c->device);
+  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
   int rc = launch_sweep(c, false, true, true, c->t + 1, c->tp + 1, gm, gext, 1);
   if (rc) return rc;
   c->t += 1; c->tp += 1;
@@ -1193,6 +1261,7 @@ int la_comm_import_step(la_ctx* c) {
   if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
   if (c->rule != LA_RULE_ADAALTER) return fail(c, LA_ESTATE, "sharding by worker is implemented for Local AdaAlter only");
   DeviceGuard guard(c->device);
+  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
   int rc = launch_sweep(c, true, true, false, c->t + 1, 1u, c->grad_kind, nullptr, 2);
   if (rc) return rc;
   c->nsync += 1; c->t += 1; c->tp = 1;
@@ -1202,6 +1271,7 @@ int la_comm_import_step(la_ctx* c) {
 int la_diagnostics(la_ctx* c, double* objective, double* replica_spread) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   DeviceGuard guard(c->device);
+  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
   if (!c->diag) {
     cudaError_t e = cudaMalloc((void**)&c->diag, 2 * sizeof(double));
     if (e != cudaSuccess) { c->diag = nullptr; cudaGetLastError(); return fail(c, LA_ENOMEM, "cudaMalloc failed: %s", cudaGetErrorString(e)); }

@@ -74,6 +74,7 @@ extern "C" int la_replica_means_static(const float* x_dev, const float* b2_dev, 
   p.X = const_cast<float*>(x_dev);  // the export pass only reads the replicas
   p.B2 = const_cast<float*>(b2_dev);
   p.xch = scratch;
+  p.xch_b_off = stride;
   p.n = n; p.stride = stride;
   p.W = W; p.W_total = W;
   const unsigned block = la::kBlockThreads;

@@ -109,7 +109,9 @@ struct SweepParams {
   uint32_t identical_workers;
   uint32_t worker_base;  // global index of local replica 0 (sharding by worker); keys use worker_base + i
   float eta, eps, sigma;
-  float* xch;            // exchange buffer [2][stride] (sums of x, sums of B^2); XCH kernels only
+  float* xch;            // XCH kernels only: where the sums of x over the replicas go to / come from ...
+  uint64_t xch_b_off;    // ... and, this many floats further, the sums of B^2 (an exchange buffer [2][stride]
+                         // has them one stride apart; replica 0's own rows, W strides)
   uint32_t W_total;      // workers over all ranks; divisor of the imported totals
 };
 
@@ -127,7 +129,7 @@ constexpr int kTreeDepth = 7;  // log2(kMaxWorkers) + 1 partial sums
 #define LA_CH 4
 #endif
 #ifndef LA_CH_V4
-#define LA_CH_V4 2
+#define LA_CH_V4 1
 #endif
 constexpr int kBlockThreads = LA_BLOCK;
 
@@ -539,7 +541,8 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
   constexpr int kChunkMax = (V == 4) ? LA_CH_V4 : LA_CH;
   constexpr int CH = (WR_ > 0) ? (WR_ < kChunkMax ? WR_ : kChunkMax) : 4;
   constexpr int kReadUnroll = (WR_ > 0) ? kMaxWorkers : 1;  // static counts: unroll fully, so that the
-  constexpr int kWriteUnroll = (W_ > 0) ? kMaxWorkers : 1;  // reduction stack is indexed by constants
+  constexpr int kWriteUnroll = (W_ > 0) ? kMaxWorkers : 4;  // reduction stack is indexed by constants; run-time
+                                                            // counts: four gradient chains in flight
   const uint32_t W = (W_ > 0) ? (uint32_t)W_ : p.W;
   const uint32_t Wr = kImport ? 1u : W;
 
@@ -577,10 +580,10 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
   const uint64_t x_base = reinterpret_cast<uint64_t>(p.X);
   const uint64_t b_delta = reinterpret_cast<uint64_t>(p.B2) - x_base;
   const uint64_t stride_bytes = p.stride * sizeof(float);
-  // read side: the replicas, or (import) the exchange buffer seen as one replica whose "B^2"
-  // sits one stride after its "x"
+  // read side: the replicas, or (import) the sums seen as one replica whose "B^2" sits
+  // xch_b_off floats after its "x"
   const uint64_t rd_base = kImport ? reinterpret_cast<uint64_t>(p.xch) : x_base;
-  const uint64_t rd_b_delta = kImport ? stride_bytes : b_delta;
+  const uint64_t rd_b_delta = kImport ? p.xch_b_off * sizeof(float) : b_delta;
 
   constexpr bool kExternal = STEP && (GM == kGradExternalF32 || GM == kGradExternalBF16);
   constexpr uint64_t kGradElem = (GM == kGradExternalBF16) ? 2 : 4;
@@ -686,7 +689,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
       if (kExport) {
         // the means are formed after the exchange, from the totals over all ranks
         st_stream<V>(p.xch + off, tree.x[0]);
-        st_stream<V>(p.xch + p.stride + off, tree.b[0]);
+        st_stream<V>(p.xch + p.xch_b_off + off, tree.b[0]);
       } else {
         // synchronisation branch of Algorithm 3: means over workers; the mean accumulator is
         // also the new stale denominator

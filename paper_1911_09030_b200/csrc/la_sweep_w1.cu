@@ -1,2 +1,6 @@
+// One replica gives a two-coordinate thread only 16 bytes of x and B^2 to fetch per group: four
+// coordinates per thread, so that enough loads are in flight to cover the memory latency.
 #define LA_W 1
+#define LA_VEC 4
+#define LA_PERIOD_VEC 2
 #include "la_sweep_inst.inc"

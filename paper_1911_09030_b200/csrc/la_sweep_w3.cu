@@ -4,6 +4,7 @@
 #define LA_VEC 4
 #define LA_CH_V4 3
 #define LA_MINB 2
+#define LA_BF16_MINB 2
 #define LA_PERIOD_VEC 2
 #define LA_PERIOD_MINB 3
 #include "la_sweep_inst.inc"

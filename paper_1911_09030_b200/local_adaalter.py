@@ -22,7 +22,7 @@ LIB_PATH = os.path.join(_HERE, "liblocal_adaalter_debug.so" if os.environ.get("L
 LA_OK, LA_EINVAL, LA_ENOMEM, LA_ECUDA, LA_ESTATE, LA_ETOOBIG, LA_EBOUNDS = 0, -1, -2, -3, -4, -5, -6
 LA_STATIC_SCRATCH_MAX_COORDS = 1048576
 LA_F32, LA_BF16 = 0, 1
-LA_FUSE_NONE, LA_FUSE_STEP_SYNC, LA_FUSE_SYNC_STEP, LA_FUSE_PERIOD = 0, 1, 2, 3
+LA_FUSE_NONE, LA_FUSE_STEP_SYNC, LA_FUSE_SYNC_STEP, LA_FUSE_PERIOD, LA_FUSE_MEAN_ONCE = 0, 1, 2, 3, 4
 LA_RULE_ADAALTER, LA_RULE_LOCAL_SGD, LA_RULE_ADAGRAD = 0, 1, 2
 LA_H_NEVER = 0xFFFFFFFF
 LA_MAX_WORKERS = 64

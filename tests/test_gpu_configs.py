@@ -146,8 +146,8 @@ def _deep_ranges(wl, nblocks=64, block=1 << 16, ends=4096, around=8):
     return merged
 
 
-DEEP_CASES = [("c2", None, (1, 3)), ("c3", None, (1, 3)), ("c5", None, (1, 3)),
-              ("c4", 1, (2,)), ("c4", 4, (0,)), ("c4", 16, (1, 3)), ("c4", 64, (2,))]
+DEEP_CASES = [("c2", None, (1, 3, 4)), ("c3", None, (1, 3, 4)), ("c5", None, (1, 3, 4)),
+              ("c4", 1, (2,)), ("c4", 4, (0, 4)), ("c4", 16, (1, 3)), ("c4", 64, (2,))]
 
 
 @pytest.mark.parametrize("name,H,fusions", DEEP_CASES, ids=[f"{n}-H{h}-f{''.join(map(str, f))}" for n, h, f in DEEP_CASES])

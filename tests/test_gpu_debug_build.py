@@ -27,7 +27,7 @@ launches = 0
 for W in (1, 3, 4, 5, 8, 16, 33):
     for n in (4, 1001, 70002):
         a = rng.uniform(0.1, 10, n).astype(np.float32); c = rng.standard_normal(n).astype(np.float32)
-        for fusion in (0, 1, 2, 3):
+        for fusion in (0, 1, 2, 3, 4):
             for bf16 in (False, True):
                 if bf16 and fusion in (0, 2):
                     continue

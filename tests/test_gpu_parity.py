@@ -25,7 +25,7 @@ def _arrays(n, seed):
 
 
 # ----------------------------------------------------------------------------- configuration 1
-@pytest.mark.parametrize("fusion", [0, 1, 2, 3])
+@pytest.mark.parametrize("fusion", [0, 1, 2, 3, 4])
 def test_config1_full(fusion):
     wl = workloads.config("c1")
     arr = wl.arrays()
@@ -59,7 +59,7 @@ def test_tails_and_worker_counts(n, W):
 def test_generic_worker_counts(W):
     n, T = 257, 9
     arr = _arrays(n, W)
-    for H, fusion in [(2, 0), (3, 1), (4, 2), (4, 3)]:
+    for H, fusion in [(2, 0), (3, 1), (4, 2), (4, 3), (2, 4), (5, 4)]:
         g, o = make_pair(n, W, 0.05, 1.0, H, "quadratic", seed=W, arrays=arr, sigma=1.0, fusion=fusion)
         g.run(T)
         o.run(T)
@@ -69,7 +69,7 @@ def test_generic_worker_counts(W):
 @pytest.mark.parametrize("grad,bf16", [("noise", False), ("noise", True), ("noise_scaled", False),
                                        ("noise_scaled", True), ("quadratic", False), ("quadratic", True),
                                        ("constant", False)])
-@pytest.mark.parametrize("fusion", [0, 1, 2, 3])
+@pytest.mark.parametrize("fusion", [0, 1, 2, 3, 4])
 def test_gradient_modes(grad, bf16, fusion):
     n, W, H, T = 70001, 4, 3, 10      # several blocks and a ragged tail
     arr = _arrays(n, 3)
@@ -88,7 +88,7 @@ def test_fused_kernels_equal_unfused_bitwise(W, H):
     n, T = 12345, 11
     arr = _arrays(n, 77)
     states = []
-    for fusion in (0, 1, 2, 3):
+    for fusion in (0, 1, 2, 3, 4):
         g = la.LocalAdaAlter([n], W, 0.1, 1.0, H)
         g.set_grad_quadratic(5, arr["a"], arr["c"], 0.2)
         g.set_fusion(fusion)
@@ -113,7 +113,7 @@ def test_fused_kernels_equal_unfused_bitwise(W, H):
 
 # ----------------------------------------------------------------------------- schedule
 @pytest.mark.parametrize("H,T", [(1, 5), (2, 5), (3, 9), (5, 5), (6, 5), (la.LA_H_NEVER, 6)])
-@pytest.mark.parametrize("fusion", [0, 1, 2, 3])
+@pytest.mark.parametrize("fusion", [0, 1, 2, 3, 4])
 def test_schedule_counters_match_oracle(H, T, fusion):
     g, o = make_pair(64, 2, 0.1, 1.0, H, "noise", seed=1, fusion=fusion)
     for _ in range(T):
@@ -146,7 +146,7 @@ def test_manual_steps_and_sync():
     assert g.get_counters() == (4, 0, 3)
 
 
-@pytest.mark.parametrize("fusion", [1, 3])
+@pytest.mark.parametrize("fusion", [1, 3, 4])
 def test_warmup_matches_oracle(fusion):
     g, o = make_pair(513, 4, 0.5, 1.0, 4, "noise", seed=8, warmup=6, b0sq=1.0, fusion=fusion)
     g.run(11); o.run(11)
@@ -393,7 +393,7 @@ def test_no_write_outside_the_arena(W, n):
     arr = _arrays(n, 9)
     g = la.LocalAdaAlter([n], W, 0.1, 1.0, 3, arena=arena, device=torch.cuda.current_device())
     g.set_grad_quadratic(4, arr["a"], arr["c"], 0.5)
-    for fusion in (0, 1, 2, 3):
+    for fusion in (0, 1, 2, 3, 4):
         g.set_fusion(fusion)
         g.run(7)
     g.set_grad_noise(4, arr["s"]); g.run(4)
@@ -501,7 +501,7 @@ def test_random_call_sequences_match_oracle(seed):
         elif op == 4 and rule != 2:                              # AdaGrad has nothing to synchronise
             g.sync(); o.sync()
         elif op == 5:
-            g.set_fusion(int(rng.integers(0, 4)))
+            g.set_fusion(int(rng.integers(0, 5)))
             g.set_launch_shape(int(rng.choice([0, 1, 7, 4096])))
         elif op == 6 and o.counters()[1] == 0:
             rule = int(rng.integers(0, 3))                       # Local AdaAlter, Local SGD, AdaGrad
@@ -556,7 +556,7 @@ def test_run_time_worker_counts_over_many_blocks(W):
     and a ragged tail, through every fusion mode."""
     n, H, T = 150001, 3, 7
     arr = _arrays(n, W)
-    for fusion in (0, 1, 2, 3):
+    for fusion in (0, 1, 2, 3, 4):
         g, o = make_pair(n, W, 0.05, 1.0, H, "noise_scaled", seed=W, arrays=arr, fusion=fusion)
         g.run(T); o.run(T)
         compare(g, o, W, TOL_RUN)
@@ -582,3 +582,42 @@ def test_noise_building_blocks_over_their_whole_domain():
     assert np.array_equal(c.cpu().numpy().view(np.uint32), oc.view(np.uint32))
     assert np.array_equal(s.cpu().numpy().view(np.uint32), os_.view(np.uint32))
     assert la.noise_tables(None, None, None) == la.LA_OK
+
+
+@pytest.mark.parametrize("W,n,H", [(4, 70002, 3), (8, 4099, 2), (16, 1000, 4), (3, 777, 5), (5, 3001, 2), (1, 513, 3), (33, 260, 2)])
+def test_mean_once_fusion_pending_sums_are_completed_on_demand(W, n, H):
+    """LA_FUSE_MEAN_ONCE keeps the result of a synchronisation as ONE copy (the sums over the workers in
+    replica 0's rows) until the next step consumes it.  Runs that end exactly on a period boundary leave
+    those sums pending; every way of looking at or touching the state must complete them first, and
+    the run must carry on from the pending state in the next call — all bitwise against the oracle."""
+    import torch
+    arr = _arrays(n, W + H)
+    g, o = make_pair(n, W, 0.05, 0.7, H, "quadratic", seed=5, arrays=arr, sigma=0.4, b0sq=0.25, fusion=4)
+    g.run(H); o.run(H)                       # ends on the boundary: sums pending
+    compare(g, o, W, TOL_RUN)                # a read completes them
+    g.run(2 * H); o.run(2 * H)               # pending again ...
+    g.run(H + 1); o.run(H + 1)               # ... and consumed by the first step of this call
+    compare(g, o, W, TOL_RUN)
+    g.run(H - 1); o.run(H - 1)               # pending
+    g.local_step(); o.local_step()           # a manual step completes them first
+    g.sync(); o.sync()
+    compare(g, o, W, TOL_RUN)
+    g.run(H); o.run(H)                       # pending
+    i = W - 1
+    x, b2, bs = g.read_state(i)
+    g.write_state(i, x, b2, bs)              # a per-worker write
+    g.run(H); o.run(H)                       # pending
+    g.set_fusion(2)                          # another fusion mode takes over from the pending state
+    g.run(2 * H + 1); o.run(2 * H + 1)
+    compare(g, o, W, TOL_RUN)
+    g.sync(); o.sync()
+    g.set_fusion(4)
+    g.run(H); o.run(H)                       # pending
+    G = np.random.default_rng(0).standard_normal((W, n)).astype(np.float32)
+    Gd = torch.from_numpy(G).cuda()
+    g.step_grads(Gd.data_ptr(), la.LA_F32); o.local_step(G)   # supplied gradients after pending sums
+    if o.counters()[1] == H:
+        o.sync()
+    compare(g, o, W, TOL_RUN)
+    st = g.get_stats()
+    assert st["launches_step_sync"] > 0 and st["launches_sync_step"] > 0
