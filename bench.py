@@ -6,11 +6,13 @@
 A "step" is one `la_run(T)` of the chosen configuration: T iterations of Algorithm 3 for all
 W workers over all N coordinates, including the synchronisations that fall in it.  The default
 workload is the largest single-GPU configuration (c5: 200 ragged tensors, 4e8 coordinates, four
-workers, bf16-rounded gradients, 13.4 GiB of state).  Prints ONE JSON line: the whole-run rate,
+workers, bf16-rounded gradients, 13.4 GiB of state), run with the per-step kernels and the
+synchronised state stored once (LA_FUSE_MEAN_ONCE).  Prints ONE JSON line: the whole-run rate,
 per-kernel durations and HBM roofline fractions of the local step (K1), the stand-alone
 synchronisation (K2) and both fusions (K3, K4), the temporal-blocking mode, the end-to-end rate
 with host buffers, the CPU oracle on the host cores, and — on one GPU — configuration 2 and the
-synchronisation-period sweep of configuration 4.  With N > 1 GPUs (torchrun) each rank runs the
+synchronisation-period sweep of configuration 4, and the by-worker layout (`--sharding worker`
+runs that layout alone, across ranks).  With N > 1 GPUs (torchrun) each rank runs the
 same configuration on its own coordinate range (coordinates never interact, so there is no
 data-path collective): weak scaling.  `--impl reference` times the CPU oracle, as it stands, on
 a bounded sample.
@@ -247,6 +249,10 @@ def workload_config(wl, args):
 # --------------------------------------------------------------------------- CUDA leg
 KERNEL_NAMES = {"local": "K1 local step", "sync": "K2 sync", "step_sync": "K3 step+sync",
                 "sync_step": "K4 sync+next step", "period": "temporal blocking"}
+# With LA_FUSE_MEAN_ONCE the two passes next to a synchronisation move about half the bytes of K3 / K4
+# (one side of the replicas is a single copy) for the same arithmetic, so they are reported apart.
+MEAN_ONCE_NAMES = {"step_sync": ("step_sums", "step t'=H storing only the sums over the workers"),
+                   "sync_step": ("means_step", "step t'=1 reading the one stored copy")}
 
 
 def per_kernel(stats, peak, leg):
@@ -381,7 +387,11 @@ def run_ours(args, wl):
     # ---- the same run again with CUDA events around every launch: per-kernel durations -------
     kernels = {}
     _, st, _ = job.timed(args.fusion, args.steps, 1, barrier, profiling=True)
-    kernels.update(per_kernel(st, peak, f"la_run, fusion {args.fusion}, {args.steps} steps"))
+    for k, v in per_kernel(st, peak, f"la_run, fusion {args.fusion}, {args.steps} steps").items():
+        if args.fusion == la.LA_FUSE_MEAN_ONCE and k in MEAN_ONCE_NAMES:
+            k, v["kernel"] = MEAN_ONCE_NAMES[k]
+            v["bound"] = "instruction issue (half the bytes of K3 / K4 for the same arithmetic)"
+        kernels[k] = v
     short = max(1, min(args.steps, 3))
     if not args.main_only:
         for fusion in (la.LA_FUSE_NONE, la.LA_FUSE_STEP_SYNC, la.LA_FUSE_SYNC_STEP):
@@ -481,6 +491,8 @@ def side_config(la, wl, peak, barrier, sampler, steps=3):
     out = {"workload": workload_config(wl, None)["workload"], "steps": steps, "ms_per_step": ms,
            "value": units / (ms * 1e-3), "unit": UNIT,
            "kernels": per_kernel(st, peak, f"la_run, fusion 1, {steps} steps")}
+    mms, _, _ = job.timed(la.LA_FUSE_MEAN_ONCE, steps, 2, barrier)
+    out["mean_once"] = {"ms_per_step": mms, "value": units / (mms * 1e-3), "unit": UNIT}
     pms, pst, pwin = job.timed(la.LA_FUSE_PERIOD, steps, 2, barrier)
     period = {"ms_per_step": pms, "steps": steps, "value": units / (pms * 1e-3), "unit": UNIT, "n_gpus": 1,
               "launches_per_step": int(pst["launches_fused"]) // steps,
@@ -492,8 +504,10 @@ def side_config(la, wl, peak, barrier, sampler, steps=3):
 
 def sync_period_sweep(la, wl, peak, barrier):
     """Configuration 4: for every synchronisation period H, one full la_run(T) unfused (K1 + K2),
-    with the step fused into its synchronisation (K3) and with the synchronisation folded into the
-    next step (K4); share of device time spent synchronising.  The single-GPU analogue of the
+    with the step fused into its synchronisation (K3), with the synchronisation folded into the
+    next step (K4), and with the synchronised state stored once (LA_FUSE_MEAN_ONCE, where the
+    passes next to a synchronisation are cheaper than a plain step); share of device time spent
+    synchronising.  The single-GPU analogue of the
     2/H communication claim of Section 4.2."""
     import copy
     rows = []
@@ -501,7 +515,9 @@ def sync_period_sweep(la, wl, peak, barrier):
         w = copy.copy(wl)
         w.H = H
         job = Job(la, w)
-        for fusion in (la.LA_FUSE_NONE, la.LA_FUSE_STEP_SYNC, la.LA_FUSE_SYNC_STEP):
+        for fusion in (la.LA_FUSE_NONE, la.LA_FUSE_STEP_SYNC, la.LA_FUSE_SYNC_STEP, la.LA_FUSE_MEAN_ONCE):
+            if fusion == la.LA_FUSE_MEAN_ONCE and H < 2:
+                continue                                    # with H = 1 it is LA_FUSE_STEP_SYNC
             job.ctx.set_fusion(fusion)
             job.ctx.run(2 * H if 2 * H < w.T else w.T)      # warm-up: two periods
             ms, st, _ = job.timed(fusion, 1, 0, barrier, profiling=True)
@@ -513,6 +529,8 @@ def sync_period_sweep(la, wl, peak, barrier):
                 for c in ("step_sync", "sync_step"):
                     if c in ker:
                         sync_ms += st[f"launches_{c}"] * max(0.0, ker[c]["ms_per_launch"] - ms_k1)
+            if fusion == la.LA_FUSE_MEAN_ONCE:
+                ker = {MEAN_ONCE_NAMES.get(c, (c,))[0]: v for c, v in ker.items()}
             rows.append({"H": H, "fusion": fusion, "T": w.T, "ms_per_run": ms,
                          "value": w.W * w.N * w.T / (ms * 1e-3),
                          "sync_share_of_device_time": sync_ms / tot if tot > 0 else None,
@@ -823,7 +841,7 @@ def main():
     ap.add_argument("--H", type=int, default=None, help="override the synchronisation period")
     ap.add_argument("--T", type=int, default=None, help="override iterations per step")
     ap.add_argument("--N", type=int, default=None, help="override the size (one flat tensor), e.g. for small ncu captures")
-    ap.add_argument("--fusion", type=int, default=1,
+    ap.add_argument("--fusion", type=int, default=4,
                     help="0 unfused, 1 step+sync, 2 sync+next step, 3 temporal blocking, 4 synchronised state stored once")
     ap.add_argument("--blocks-per-sm", type=int, default=0)
     ap.add_argument("--sharding", default="coordinate", choices=["coordinate", "worker"],
