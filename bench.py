@@ -39,11 +39,14 @@ FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 # Figures taken from the ncu captures summarised in profiles/, valid only for the kernel sources
 # they were taken on (KERNEL_HASH_AT_CAPTURE):
-#   NCU_TRAFFIC_BYTES             dram__bytes_read.sum + dram__bytes_write.sum per K1 launch
+#   NCU_TRAFFIC_BYTES             dram__bytes_read.sum + dram__bytes_write.sum per K1 launch.  c2: captured at
+#                                 full size.  c5: captured at N = 2^25 (1.5 GiB of state; the full 13.4 GiB is too
+#                                 much to save and restore around ncu's replay passes) and scaled by
+#                                 400 007 886 / 2^25 — every byte is touched once, so traffic grows with N.
 #   PERIOD_LANE_INSTR_PER_UPDATE  smsp__inst_executed.sum x 32 / updates per la_period launch
-KERNEL_HASH_AT_CAPTURE = "f7182c402edd33c4"
-NCU_TRAFFIC_BYTES = {"c2": 2.2240e9}
-PERIOD_LANE_INSTR_PER_UPDATE = {"c2": 50.5}
+KERNEL_HASH_AT_CAPTURE = "381d43966e24dce2"
+NCU_TRAFFIC_BYTES = {"c2": 2.2234e9, "c5": 29.741e9}
+PERIOD_LANE_INSTR_PER_UPDATE = {"c2": 43.15}
 
 
 def kernel_source_hash():
@@ -54,10 +57,12 @@ def kernel_source_hash():
     for name in ("grad_source.cuh", "la_sweep.cuh", "la_period.cuh", "la_exchange.cuh"):
         with open(os.path.join(d, name), "rb") as fh:
             h.update(fh.read())
-    with open(os.path.join(d, "la_sweep_inst.inc")) as fh:
-        for line in fh:
-            if line.startswith("#define LA_"):
-                h.update(line.encode())
+    import glob
+    for path in [os.path.join(d, "la_sweep_inst.inc")] + sorted(glob.glob(os.path.join(d, "la_sweep_w*.cu"))):
+        with open(path) as fh:
+            for line in fh:
+                if line.startswith("#define LA_"):
+                    h.update(line.encode())
     return h.hexdigest()[:16]
 
 
