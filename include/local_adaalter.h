@@ -181,6 +181,34 @@ int la_sync(la_ctx* ctx);
  * kernels; the state afterwards is bitwise that of the unfused sequence. */
 int la_run(la_ctx* ctx, uint64_t T);
 
+/* A whole job from and to host memory in one call, pipelined: equivalent to
+ *   la_set_init(x0_host, b0sq as last set); the la_set_grad_* upload of the arrays given here;
+ *   la_run(T); la_read_state(worker, x_host, b2_host, bs_host)
+ * with the same bits in the outputs, in the device state and in the counters afterwards, but the
+ * coordinates are cut into `chunks` ranges (0 = 16) and the upload of one range, the T iterations
+ * of the previous one and the download of the one before overlap on three streams.  This is legal
+ * because Algorithm 3 has only coordinate-wise operations and a per-coordinate mean over workers.
+ * Host buffers hold N floats each and should be pinned (page-locked) for the copies to overlap.
+ *   x0_host              initial iterate, or NULL for zeros
+ *   a_host, c_host       quadratic gradient source: both or neither (NULL keeps the arrays on the device)
+ *   s_host               scale array of the noise / constant sources, or NULL (keeps what is there)
+ *   worker               whose x and B^2 are read back
+ *   x_host, b2_host, bs_host   outputs, any may be NULL
+ * The gradient source, its seed and sigma, the rule, the fusion mode and H are those of the
+ * context.  Returns after the outputs are complete.  Two copy streams and 2 * chunks events are
+ * created on the first call and live until la_destroy. */
+typedef struct la_stream_io {
+  const float* x0_host;
+  const float* a_host;
+  const float* c_host;
+  const float* s_host;
+  uint32_t worker;
+  float* x_host;
+  float* b2_host;
+  float* bs_host;
+} la_stream_io;
+int la_run_streamed(la_ctx* ctx, uint64_t T, const la_stream_io* io, uint32_t chunks);
+
 /* ---- state access (synchronises the stream) ------------------------------------
  * Copy worker `worker`'s x and B^2 and the shared stale accumulator to host buffers of N floats
  * each, in packed tensor order.  Any pointer may be NULL. */

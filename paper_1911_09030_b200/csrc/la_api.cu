@@ -68,10 +68,11 @@ PeriodKernel lookup_period(int W, int gm, bool bf16, bool post) {
 
 constexpr int kExchangeVec = 2;  // coordinates per thread in the combine kernel
 
+// Coordinates [0, count) of every replica: x0 (zeros from n on, or everywhere without x0), b0sq.
 __global__ void la_fill(float* X, float* B2, float* Bs, const float* x0, float b0sq, uint64_t stride,
-                        uint64_t n, uint32_t W) {
+                        uint64_t n, uint64_t count, uint32_t W) {
   const uint64_t nthreads = (uint64_t)gridDim.x * blockDim.x;
-  for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < stride; j += nthreads) {
+  for (uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; j < count; j += nthreads) {
     const float v = (x0 != nullptr && j < n) ? x0[j] : 0.0f;
     for (uint32_t i = 0; i < W; ++i) {
       X[(uint64_t)i * stride + j] = v;
@@ -214,6 +215,10 @@ struct la_ctx {
   float* peerS[la::kMaxRanks] = {};
   void* ipc_opened[la::kMaxRanks] = {};
   double* diag = nullptr;  // two doubles for la_diagnostics, allocated on its first call
+  // la_run_streamed: copy streams and per-chunk events, created on first use
+  cudaStream_t copy_in = nullptr, copy_out = nullptr;
+  std::vector<cudaEvent_t> ev_in, ev_done;
+  cudaEvent_t ev_idle = nullptr;
   // checked build (LA_DEBUG): device status words the kernels report address violations into,
   // and a test knob that makes the kernels treat the last `dbg_narrow` bytes of the arena as foreign
   unsigned long long* dbg_status = nullptr;
@@ -526,12 +531,14 @@ int upload_padded(la_ctx* c, float* dst, const float* src_host, float pad) {
   return LA_OK;
 }
 
-int do_fill(la_ctx* c, const float* x0_dev) {
+// count = 0: the whole arrays up to the replica stride (padding included).
+int do_fill(la_ctx* c, const float* x0_dev, uint64_t count = 0) {
   const unsigned block = 256;
-  uint64_t blocks = (c->stride + block - 1) / block;
+  if (count == 0) count = c->stride;
+  uint64_t blocks = (count + block - 1) / block;
   const uint64_t cap = (uint64_t)c->num_sms * 16;
   if (blocks > cap) blocks = cap;
-  la::la_fill<<<(unsigned)blocks, block, 0, c->stream>>>(c->X, c->B2, c->Bs, x0_dev, c->b0sq, c->stride, c->N, c->W);
+  la::la_fill<<<(unsigned)blocks, block, 0, c->stream>>>(c->X, c->B2, c->Bs, x0_dev, c->b0sq, c->stride, c->N, count, c->W);
   LA_CUDA(c, cudaGetLastError());
   c->stats.launches_other++;
   return LA_OK;
@@ -675,6 +682,11 @@ void la_destroy(la_ctx* c) {
   if (c->S) cudaFree(c->S);
   if (c->diag) cudaFree(c->diag);
   if (c->dbg_status) cudaFree(c->dbg_status);
+  for (auto e : c->ev_in) cudaEventDestroy(e);
+  for (auto e : c->ev_done) cudaEventDestroy(e);
+  if (c->ev_idle) cudaEventDestroy(c->ev_idle);
+  if (c->copy_in) cudaStreamDestroy(c->copy_in);
+  if (c->copy_out) cudaStreamDestroy(c->copy_out);
   if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
   if (c->sched) cudaFree(c->sched);
   if (c->owns_arena && c->arena) cudaFree(c->arena);
@@ -838,8 +850,25 @@ int la_step_grads(la_ctx* c, const void* g_dev, int dtype) {
   if (dtype != LA_F32 && dtype != LA_BF16) return fail(c, LA_EINVAL, "dtype must be LA_F32 or LA_BF16");
   if (c->rule == LA_RULE_ADAGRAD) return la_local_step_grads(c, g_dev, dtype);  // Algorithm 1: one pass is the whole iteration
   DeviceGuard guard(c->device);
-  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
   const int gm = dtype == LA_F32 ? la::kGradExternalF32 : la::kGradExternalBF16;
+  if (c->fusion == LA_FUSE_MEAN_ONCE && c->rule == LA_RULE_ADAALTER && c->H >= 2u) {
+    // the synchronised state is stored once (see run_steps): sums out at t' = H, one copy in at t' = 1
+    if (c->sums_in_replica0) {
+      int rc = launch_sweep(c, true, true, false, c->t + 1, 1u, gm, g_dev, 2, true);
+      if (rc) return rc;
+      c->sums_in_replica0 = false;
+      c->t += 1; c->tp = 1;
+      return LA_OK;
+    }
+    if (c->tp + 1 == c->H) {
+      int rc = launch_sweep(c, false, true, true, c->t + 1, c->tp + 1, gm, g_dev, 1, true);
+      if (rc) return rc;
+      c->sums_in_replica0 = true;
+      c->t += 1; c->tp = 0; c->nsync += 1;
+      return LA_OK;
+    }
+  }
+  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
   const bool closes = (c->tp + 1 == c->H);
   if (closes && c->fusion != LA_FUSE_NONE) {
     int rc = launch_sweep(c, false, true, true, c->t + 1, c->tp + 1, gm, g_dev);  // step and its sync in one pass
@@ -1041,6 +1070,85 @@ static int run_steps(la_ctx* c, uint64_t T) {
     }
   }
   return LA_OK;
+}
+
+// ---- a whole job from and to host memory, pipelined over coordinate ranges --------------------
+// Algorithm 3 never mixes coordinates, so [upload, T iterations, download] of one coordinate range
+// is independent of every other range: while range k computes on the context's stream, range k+1
+// is uploaded on a second stream and range k-1 downloaded on a third.  During a range the
+// context simply points at that part of its arrays (same replica stride, shifted coordinate base).
+int la_run_streamed(la_ctx* c, uint64_t T, const la_stream_io* io, uint32_t chunks) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!io) return fail(c, LA_EINVAL, "io is NULL");
+  if (io->worker >= c->W) return fail(c, LA_EINVAL, "worker %u out of range (W=%u)", io->worker, c->W);
+  if (c->grad_kind == la::kGradQuadratic && (!io->a_host != !io->c_host))
+    return fail(c, LA_EINVAL, "a_host and c_host come together");
+  if (chunks == 0) chunks = 16;
+  if (chunks > 4096) chunks = 4096;
+  DeviceGuard guard(c->device);
+  if (!c->copy_in) LA_CUDA(c, cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking));
+  if (!c->copy_out) LA_CUDA(c, cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking));
+  if (!c->ev_idle) LA_CUDA(c, cudaEventCreateWithFlags(&c->ev_idle, cudaEventDisableTiming));
+  while (c->ev_in.size() < chunks) {
+    cudaEvent_t a = nullptr, b = nullptr;
+    LA_CUDA(c, cudaEventCreateWithFlags(&a, cudaEventDisableTiming));
+    c->ev_in.push_back(a);
+    LA_CUDA(c, cudaEventCreateWithFlags(&b, cudaEventDisableTiming));
+    c->ev_done.push_back(b);
+  }
+  // the uploads overwrite the state: whatever the context's stream still does comes first
+  LA_CUDA(c, cudaEventRecord(c->ev_idle, c->stream));
+  LA_CUDA(c, cudaStreamWaitEvent(c->copy_in, c->ev_idle, 0));
+
+  struct View { float *X, *B2, *Bs, *pa, *pc, *ps; uint64_t N, j_base; } full{c->X, c->B2, c->Bs, c->pa, c->pc, c->ps, c->N, c->j_base};
+  const uint64_t per = round_up((full.N + chunks - 1) / chunks, 256);  // whole 1 KiB units: vector accesses stay aligned
+  c->shared_iterate = false;
+  c->sums_in_replica0 = false;
+  int rc = LA_OK;
+  uint32_t k = 0;
+  for (uint64_t j0 = 0; j0 < full.N && rc == LA_OK; j0 += per, ++k) {
+    const uint64_t n = (full.N - j0 < per) ? full.N - j0 : per;
+    const bool last = (j0 + n == full.N);
+    const uint64_t span = last ? c->stride - j0 : n;  // the last range also owns the padding up to the stride
+    const size_t bytes = n * sizeof(float), tail = (span - n) * sizeof(float);
+    auto up = [&](float* dst, const float* src) -> cudaError_t {
+      cudaError_t e = cudaMemcpyAsync(dst + j0, src + j0, bytes, cudaMemcpyHostToDevice, c->copy_in);
+      if (e == cudaSuccess && tail) e = cudaMemsetAsync(dst + j0 + n, 0, tail, c->copy_in);
+      return e;
+    };
+    cudaError_t e = cudaSuccess;
+    if (io->x0_host) e = cudaMemcpyAsync(full.X + j0, io->x0_host + j0, bytes, cudaMemcpyHostToDevice, c->copy_in);  // staged in replica 0
+    if (e == cudaSuccess && io->a_host) e = up(full.pa, io->a_host);
+    if (e == cudaSuccess && io->c_host) e = up(full.pc, io->c_host);
+    if (e == cudaSuccess && io->s_host) e = up(full.ps, io->s_host);
+    if (e == cudaSuccess) e = cudaEventRecord(c->ev_in[k], c->copy_in);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(c->stream, c->ev_in[k], 0);
+    if (e != cudaSuccess) { rc = fail(c, LA_ECUDA, "upload of coordinate range %u failed: %s", k, cudaGetErrorString(e)); break; }
+
+    c->X = full.X + j0; c->B2 = full.B2 + j0; c->Bs = full.Bs + j0;
+    c->pa = full.pa + j0; c->pc = full.pc + j0; c->ps = full.ps + j0;
+    c->N = n; c->j_base = full.j_base + j0;
+    c->t = 0; c->tp = 0; c->nsync = 0;
+    rc = do_fill(c, io->x0_host ? c->X : nullptr, span);
+    if (rc == LA_OK) rc = run_steps(c, T);
+    if (rc == LA_OK) rc = import_pending_sums(c);
+    if (rc != LA_OK) break;
+    e = cudaEventRecord(c->ev_done[k], c->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(c->copy_out, c->ev_done[k], 0);
+    const uint64_t row = (uint64_t)(c->shared_iterate ? 0u : io->worker) * c->stride;
+    if (e == cudaSuccess && io->x_host) e = cudaMemcpyAsync(io->x_host + j0, c->X + row, bytes, cudaMemcpyDeviceToHost, c->copy_out);
+    if (e == cudaSuccess && io->b2_host) e = cudaMemcpyAsync(io->b2_host + j0, c->B2 + row, bytes, cudaMemcpyDeviceToHost, c->copy_out);
+    if (e == cudaSuccess && io->bs_host) e = cudaMemcpyAsync(io->bs_host + j0, c->Bs, bytes, cudaMemcpyDeviceToHost, c->copy_out);
+    if (e != cudaSuccess) { rc = fail(c, LA_ECUDA, "download of coordinate range %u failed: %s", k, cudaGetErrorString(e)); break; }
+  }
+  c->X = full.X; c->B2 = full.B2; c->Bs = full.Bs; c->pa = full.pa; c->pc = full.pc; c->ps = full.ps;
+  c->N = full.N; c->j_base = full.j_base;
+  if (io->s_host) c->has_s = true;
+  // the call returns with the outputs complete and the state resident, like la_read_state
+  cudaError_t e1 = cudaStreamSynchronize(c->copy_out), e2 = cudaStreamSynchronize(c->stream);
+  if (rc != LA_OK) return rc;
+  if (e1 != cudaSuccess || e2 != cudaSuccess) return fail(c, LA_ECUDA, "stream synchronisation failed: %s", cudaGetErrorString(e1 != cudaSuccess ? e1 : e2));
+  return debug_poll(c);
 }
 
 // ---- state access ----------------------------------------------------------------------------

@@ -585,7 +585,9 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
   const uint64_t rd_base = kImport ? reinterpret_cast<uint64_t>(p.xch) : x_base;
   const uint64_t rd_b_delta = kImport ? p.xch_b_off * sizeof(float) : b_delta;
 
-  constexpr bool kExternal = STEP && (GM == kGradExternalF32 || GM == kGradExternalBF16);
+  constexpr bool kSupplied = STEP && (GM == kGradExternalF32 || GM == kGradExternalBF16);
+  constexpr bool kExternal = kSupplied && !PRE;  // table rows fetched in the replica pipeline; a step that follows an
+                                                 // average (PRE) fetches them in its write loop instead
   constexpr uint64_t kGradElem = (GM == kGradExternalBF16) ? 2 : 4;
   const uint64_t g_base = reinterpret_cast<uint64_t>(p.gext);
   const uint64_t g_row_bytes = p.n * kGradElem;
@@ -703,9 +705,17 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
           // first step of the next period: every replica starts from the mean, t' = 1
           if (ACC) r = step_size<V>(bm, q, eta_t);
 #pragma unroll kWriteUnroll
+          uint64_t gw_addr = g_base + off * kGradElem;  // supplied gradients: row i of the table, this group
           for (uint32_t i = 0; i < W; ++i) {
             Vec<V> xv = xm, bv = bm;
-            const Vec<V> g = gradient<GM, BF16, V>(p, in, xv, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
+            Vec<V> g;
+            if (kSupplied) {
+              GradChunk<V, 1> gc;
+              load_grads<GM, V, 1>(gc, p, gw_addr, g_row_bytes, W, i, off);
+              g = gc.g[0];
+            } else {
+              g = gradient<GM, BF16, V>(p, in, xv, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
+            }
             apply<V, ACC>(r, g, xv, bv);
             store_replica<V, ACC>(st_addr, b_delta, stride_bytes, xv, bv
                                   LA_DBG_ARG(x_base + off * sizeof(float) + (uint64_t)i * stride_bytes));

@@ -46,6 +46,11 @@ class la_stats(C.Structure):
                 ("bytes_step_sync", C.c_double), ("bytes_sync_step", C.c_double), ("bytes_period", C.c_double)]
 
 
+class la_stream_io(C.Structure):
+    _fields_ = [("x0_host", C.c_void_p), ("a_host", C.c_void_p), ("c_host", C.c_void_p), ("s_host", C.c_void_p),
+                ("worker", C.c_uint32), ("x_host", C.c_void_p), ("b2_host", C.c_void_p), ("bs_host", C.c_void_p)]
+
+
 _lib = None
 
 
@@ -103,6 +108,7 @@ def lib() -> C.CDLL:
             "la_stream_sync": [vp],
             "la_noise_tables": [vp, vp, vp, vp],
             "la_replica_means_static": [vp, vp, u32, u64, u64, vp, vp, vp],
+            "la_run_streamed": [vp, u64, C.POINTER(la_stream_io), u32],
             "la_debug_build": [],
             "la_debug_narrow": [vp, u64],
         }
@@ -294,6 +300,22 @@ class LocalAdaAlter:
 
     def run(self, T):
         self._ck(self.L.la_run(self.h, int(T)))
+
+    def run_streamed(self, T, worker=0, x0=None, a=None, c=None, s=None, x_out=None, b2_out=None, bs_out=None,
+                     chunks=0):
+        """`la_run_streamed`: init from host arrays, T iterations, read-back of one worker — pipelined
+        over coordinate ranges.  Arrays are float32 numpy arrays or CPU torch tensors (pinned for overlap)
+        of N elements; outputs are written in place."""
+        keep, io = [], la_stream_io()
+        for name, arr in (("x0_host", x0), ("a_host", a), ("c_host", c), ("s_host", s),
+                          ("x_host", x_out), ("b2_host", b2_out), ("bs_host", bs_out)):
+            k, ptr = _as_f32(arr, self.N, name)
+            if arr is not None and name in ("x_host", "b2_host", "bs_host") and k is not arr:
+                raise ValueError(f"{name}: outputs must be contiguous float32 buffers of {self.N} elements")
+            keep.append(k)
+            setattr(io, name, ptr.value if ptr is not None else None)
+        io.worker = int(worker)
+        self._ck(self.L.la_run_streamed(self.h, int(T), C.byref(io), int(chunks)))
 
     # ------------------------------------------------------------------ state
     def read_state(self, worker, want=("x", "b2", "bs"), out=None):

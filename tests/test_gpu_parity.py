@@ -621,3 +621,39 @@ def test_mean_once_fusion_pending_sums_are_completed_on_demand(W, n, H):
     compare(g, o, W, TOL_RUN)
     st = g.get_stats()
     assert st["launches_step_sync"] > 0 and st["launches_sync_step"] > 0
+
+
+@pytest.mark.parametrize("W,n,H,T,grad,fusion,chunks,bf16", [
+    (4, 70001, 3, 10, "quadratic", 4, 3, True), (8, 5000, 2, 7, "noise_scaled", 1, 16, False),
+    (3, 1025, 4, 8, "noise", 3, 5, False), (16, 300, 1, 3, "quadratic", 2, 1, False),
+    (5, 40000, 5, 11, "quadratic", 0, 7, False), (1, 2049, 2, 4, "noise_scaled", 4, 2, False)])
+def test_streamed_run_equals_upload_run_download(W, n, H, T, grad, fusion, chunks, bf16):
+    """la_run_streamed pipelines [upload, T iterations, download] over coordinate ranges; outputs,
+    device state and counters must be those of la_set_init + la_set_grad_* + la_run + la_read_state,
+    i.e. the oracle's, bitwise — also when it is called again on a used context, and for a worker
+    other than 0."""
+    import torch
+    rng = np.random.default_rng(n)
+    arr = _arrays(n, W)
+    x0 = rng.standard_normal(n).astype(np.float32)
+    g, o = make_pair(n, W, 0.05, 0.7, H, grad, seed=4, arrays=arr, sigma=0.4, bf16=bf16, fusion=fusion, b0sq=0.5, x0=x0)
+    o.run(T)
+    g.run(3)                                                    # a used context: the call re-initialises it
+    pin = lambda a: torch.from_numpy(a).pin_memory()
+    outs = {k: torch.empty(n, dtype=torch.float32).pin_memory() for k in ("x", "b2", "bs")}
+    w = W - 1
+    kw = {"a": pin(arr["a"]), "c": pin(arr["c"])} if grad == "quadratic" else ({"s": pin(arr["s"])} if grad == "noise_scaled" else {})
+    for rep in range(2):
+        g.run_streamed(T, worker=w, x0=pin(x0), x_out=outs["x"], b2_out=outs["b2"], bs_out=outs["bs"], chunks=chunks, **kw)
+        assert g.get_counters() == o.counters()
+        for got, ref in zip((outs["x"], outs["b2"], outs["bs"]), o.read(w)):
+            assert np.array_equal(got.numpy().view(np.uint32), ref.view(np.uint32))
+    compare(g, o, W, TOL_RUN)                                   # the resident state as well
+    g.run(H + 1); o.run(H + 1)                                  # and the run carries on from it
+    compare(g, o, W, TOL_RUN)
+    x_np = np.empty(n, np.float32)                              # pageable memory works too (without overlap)
+    g.run_streamed(T, worker=0, x0=x0, x_out=x_np, chunks=chunks,
+                   **{k: v.numpy() for k, v in kw.items()})
+    o2 = make_pair(n, W, 0.05, 0.7, H, grad, seed=4, arrays=arr, sigma=0.4, bf16=bf16, fusion=fusion, b0sq=0.5, x0=x0)[1]
+    o2.run(T)
+    assert np.array_equal(x_np.view(np.uint32), o2.read(0)[0].view(np.uint32))
