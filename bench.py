@@ -44,9 +44,9 @@ NOMINAL_HBM_GBS = 8000.0
 #                                 much to save and restore around ncu's replay passes) and scaled by
 #                                 400 007 886 / 2^25 — every byte is touched once, so traffic grows with N.
 #   PERIOD_LANE_INSTR_PER_UPDATE  smsp__inst_executed.sum x 32 / updates per la_period launch
-KERNEL_HASH_AT_CAPTURE = "381d43966e24dce2"
-NCU_TRAFFIC_BYTES = {"c2": 2.2234e9, "c5": 29.741e9}
-PERIOD_LANE_INSTR_PER_UPDATE = {"c2": 43.15}
+KERNEL_HASH_AT_CAPTURE = "db7a1f5f7d0d01e8"
+NCU_TRAFFIC_BYTES = {"c2": 2.2235e9, "c5": 29.742e9}
+PERIOD_LANE_INSTR_PER_UPDATE = {"c2": 43.15, "c5": 50.89}   # c5: captured at N = 2^25 (the count per update does not depend on N)
 
 
 def kernel_source_hash():
@@ -743,14 +743,17 @@ def run_kernel_report(args):
     peak, peak_kind = measured_peak()
     rows = []
 
-    def classes(ctx, W, what):
+    def classes(ctx, W, what, once=False):
         st = ctx.get_stats(reset=True)
         for cls in ("local", "sync", "step_sync", "sync_step"):
             n = st[f"launches_{cls}"]
+            if once and cls not in MEAN_ONCE_NAMES:
+                continue
             if n and st[f"ms_{cls}"] > 0:
                 ms = st[f"ms_{cls}"] / n
                 gbs = st[f"bytes_{cls}"] / n / (ms * 1e-3) / 1e9
-                rows.append({"W": W, "N": ctx.N, "gradients": what, "kernel": KERNEL_NAMES[cls], "launches": int(n),
+                rows.append({"W": W, "N": ctx.N, "gradients": what,
+                             "kernel": MEAN_ONCE_NAMES[cls][1] if once else KERNEL_NAMES[cls], "launches": int(n),
                              "us_per_launch": 1e3 * ms, "GBps": gbs, "frac": gbs / peak})
 
     for W in args.workers:
@@ -784,6 +787,18 @@ def run_kernel_report(args):
                     ctx.step_grads(G.data_ptr(), dtype)
                 ctx.set_profiling(False)
                 classes(ctx, W, name)
+                ctx.sync()
+                ctx.set_fusion(la.LA_FUSE_MEAN_ONCE)      # the same table with the synchronised state stored once
+                for _ in range(8):
+                    ctx.step_grads(G.data_ptr(), dtype)
+                ctx.sync_stream()
+                ctx.get_stats(reset=True)
+                ctx.set_profiling(True)
+                for _ in range(24):
+                    ctx.step_grads(G.data_ptr(), dtype)
+                ctx.set_profiling(False)
+                classes(ctx, W, name, once=True)
+                ctx.sync()
                 del G
         ctx.close()
         torch.cuda.empty_cache()

@@ -52,7 +52,7 @@ for W, n in ((4, 4096), (8, 1001), (5, 70002)):
         for rule in (la.LA_RULE_ADAALTER, la.LA_RULE_ADAGRAD):
             g = la.LocalAdaAlter([n], W, 0.1, 1.0, 2)
             g.set_rule(rule)
-            g.set_fusion(1)
+            g.set_fusion(1 if W == 8 else 4)
             for t in range(5):
                 G = torch.randn(W, n, device="cuda").to(tdt)
                 g.step_grads(G.data_ptr(), dtype)

@@ -253,7 +253,8 @@ def test_supplied_gradients_match_oracle(dtype, n):
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("W,n,H,fusion", [(4, 70002, 3, 1), (8, 4098, 2, 0), (16, 1000, 4, 1), (3, 777, 2, 1),
-                                           (2, 12, 1, 1), (5, 4100, 3, 2)])
+                                           (2, 12, 1, 1), (5, 4100, 3, 2), (4, 70002, 3, 4), (8, 4098, 2, 4),
+                                           (3, 777, 5, 4), (1, 2052, 2, 4), (33, 260, 3, 4), (2, 12, 1, 4)])
 def test_step_grads_full_iteration(dtype, W, n, H, fusion):
     """la_step_grads = local step + the synchronisation when it is due (fused or not); even n takes
     the vector loads, odd n the scalar ones; a table offset by one element is mis-aligned."""
@@ -281,6 +282,9 @@ def test_step_grads_full_iteration(dtype, W, n, H, fusion):
     st = g.get_stats()
     if fusion == 0:
         assert st["launches_fused"] == 0 and st["launches_sync"] == T // H
+    elif fusion == 4 and H >= 2:
+        # sums out at every t' = H, one copy in at every following t' = 1; the final read completed pending sums
+        assert st["launches_step_sync"] == T // H and st["launches_sync_step"] == (T - 1) // H
     else:
         assert st["launches_fused"] == T // H and st["launches_sync"] == 0
 
