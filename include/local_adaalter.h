@@ -59,8 +59,9 @@ enum { LA_FUSE_NONE = 0, LA_FUSE_STEP_SYNC = 1, /* la_run: step t'=H and its syn
                                                    its y, A^2 over the workers (into replica 0's rows) and the
                                                    step t'=1 that follows reads that one copy; per period one
                                                    write and one read of W-1 replicas fewer than LA_FUSE_STEP_SYNC.
-                                                   Generated gradients, Local AdaAlter, H >= 2 (otherwise it
-                                                   behaves as LA_FUSE_STEP_SYNC).  Between the two steps, also
+                                                   la_run (generated gradients) and la_step_grads (supplied
+                                                   ones), Local AdaAlter, H >= 2 (otherwise it behaves as
+                                                   LA_FUSE_STEP_SYNC).  Between the two steps, also
                                                    across calls, the means are pending; every call that looks
                                                    at or changes the state completes them first. */
 enum { LA_RULE_ADAALTER = 0,  /* Algorithm 3, Local AdaAlter (default) */
