@@ -24,7 +24,7 @@ from oracle.oracle import Oracle
 assert la.debug_build(), "the checked library was not loaded"
 rng = np.random.default_rng(3)
 launches = 0
-for W in (1, 3, 4, 5, 8, 16, 33):
+for W in (1, 3, 4, 5, 8, 16, 33, 48):
     for n in (4, 1001, 70002):
         a = rng.uniform(0.1, 10, n).astype(np.float32); c = rng.standard_normal(n).astype(np.float32)
         for fusion in (0, 1, 2, 3, 4):

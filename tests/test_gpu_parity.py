@@ -55,7 +55,7 @@ def test_tails_and_worker_counts(n, W):
         g.close()
 
 
-@pytest.mark.parametrize("W", [5, 6, 7, 11, 13, 64])
+@pytest.mark.parametrize("W", [5, 6, 7, 11, 13, 24, 32, 40, 48, 64])
 def test_generic_worker_counts(W):
     n, T = 257, 9
     arr = _arrays(n, W)
@@ -661,3 +661,33 @@ def test_streamed_run_equals_upload_run_download(W, n, H, T, grad, fusion, chunk
     o2 = make_pair(n, W, 0.05, 0.7, H, grad, seed=4, arrays=arr, sigma=0.4, bf16=bf16, fusion=fusion, b0sq=0.5, x0=x0)[1]
     o2.run(T)
     assert np.array_equal(x_np.view(np.uint32), o2.read(0)[0].view(np.uint32))
+
+
+@pytest.mark.parametrize("W", [32, 48, 64])
+def test_worker_counts_of_whole_tiles(W):
+    """W = 32, 48, 64 (run-time worker counts made of whole tiles of 16 replicas, summed by the
+    constant-index tree and pushed into the run-time counter as aligned blocks): the result is the
+    adjacent-pair tree over all W workers, bitwise, for the stand-alone synchronisation, both
+    fusions, supplied gradient tables and manual call sequences."""
+    import torch
+    n, H = 1537, 3
+    arr = _arrays(n, W)
+    for fusion in (0, 1, 2):
+        g, o = make_pair(n, W, 0.05, 0.7, H, "noise_scaled", seed=W, arrays=arr, fusion=fusion, b0sq=0.5)
+        g.run(2 * H + 1); o.run(2 * H + 1)
+        g.sync(); o.sync()                                         # a manual synchronisation inside a period
+        g.run(H); o.run(H)
+        compare(g, o, W, TOL_RUN)
+        st = g.get_stats()
+        assert st["launches_sync"] + st["launches_fused"] >= 3
+    g, o = make_pair(n, W, 0.05, 0.7, H, "noise", seed=1, fusion=1)
+    rng = np.random.default_rng(W)
+    for dtype, tdt in ((la.LA_F32, torch.float32), (la.LA_BF16, torch.bfloat16)):
+        for t in range(H + 1):
+            G = torch.from_numpy(rng.standard_normal((W, n)).astype(np.float32)).to(tdt)
+            Gd = G.cuda()
+            g.step_grads(Gd.data_ptr(), dtype); o.local_step(G.float().numpy())
+            if o.counters()[1] == H:
+                o.sync()
+            g.sync_stream()
+    compare(g, o, W, TOL_RUN)
