@@ -128,6 +128,10 @@ class OracleEngine:
         self.buf[self.n:] = torch.from_numpy(self._tree(bs))
     def combine(self): raise AssertionError("peer exchange needs device memory")
     def buffer_tensor(self): return self.buf
+    def step_export(self):          # the closing step, then its sums (the CUDA engine never stores y, A^2)
+        self.o.local_step(); self.export()
+    def import_step(self):          # the means, then the first step of the next period
+        self.import_(); self.o.local_step()
     def import_(self):
         w = np.float32(self.W_total)
         xm = self.buf[:self.n].numpy() / w
@@ -146,8 +150,11 @@ a = rng.uniform(0.1, 10, n).astype(np.float32); c = rng.standard_normal(n).astyp
 o = Oracle(n, W_local, 0.1, 1.0, 0xFFFFFFFF)
 o.set_grad_quadratic(9, a, c, 0.3)
 o.set_worker_base(rank * W_local)
-job = WorkerShardedJob(OracleEngine(o, W_local, W_total, n), H, exchange="allreduce", dist=dist)
-job.run(T)
+job = WorkerShardedJob(OracleEngine(o, W_local, W_total, n), H, exchange="allreduce", dist=dist,
+                       fused=os.environ.get("LA_FUSED") == "1")
+job.run(4)                      # ends inside a period; the schedule carries on in the next call
+job.run(T - 4)
+assert job.exchange_seconds > 0.0
 mine = np.stack([o.read(i)[0] for i in range(W_local)])
 parts = [None] * world
 dist.all_gather_object(parts, (rank, mine, o.counters(), job.syncs))
@@ -165,12 +172,14 @@ dist.destroy_process_group()
 '''
 
 
-def test_two_gloo_ranks_sharded_by_worker(tmp_path):
-    """The by-worker choreography (export, all-reduce, import, counters) on two CPU ranks with
-    an oracle-backed engine equals the single-process oracle with W_total workers, bitwise."""
+@pytest.mark.parametrize("fused", [False, True])
+def test_two_gloo_ranks_sharded_by_worker(tmp_path, fused):
+    """The by-worker choreography (export, all-reduce, import, counters; also with the steps next to
+    a synchronisation fused into the exchange) on two CPU ranks with an oracle-backed engine equals
+    the single-process oracle with W_total workers, bitwise."""
     script = tmp_path / "by_worker.py"
     script.write_text(WORKER_BY_WORKER)
-    env = dict(os.environ, LA_ROOT=ROOT, MASTER_ADDR="127.0.0.1")
+    env = dict(os.environ, LA_ROOT=ROOT, MASTER_ADDR="127.0.0.1", LA_FUSED="1" if fused else "0")
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
            "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), str(script)]
     r = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=300)
