@@ -27,6 +27,8 @@ SweepKernel lookup_sweep_w16(int, int, bool, bool, bool, bool, int);
 SweepKernel lookup_sweep_w3(int, int, bool, bool, bool, bool, int);
 SweepKernel lookup_sweep_w6(int, int, bool, bool, bool, bool, int);
 SweepKernel lookup_sweep_w12(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w32(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w64(int, int, bool, bool, bool, bool, int);
 
 SweepKernel lookup_sweep(int W, int rule, int gm, bool bf16, bool pre, bool step, bool post, int xch) {
   switch (W) {
@@ -38,6 +40,8 @@ SweepKernel lookup_sweep(int W, int rule, int gm, bool bf16, bool pre, bool step
     case 3: return lookup_sweep_w3(rule, gm, bf16, pre, step, post, xch);
     case 6: return lookup_sweep_w6(rule, gm, bf16, pre, step, post, xch);
     case 12: return lookup_sweep_w12(rule, gm, bf16, pre, step, post, xch);
+    case 32: return lookup_sweep_w32(rule, gm, bf16, pre, step, post, xch);
+    case 64: return lookup_sweep_w64(rule, gm, bf16, pre, step, post, xch);
     default: return lookup_sweep_w0(rule, gm, bf16, pre, step, post, xch);
   }
 }
@@ -51,6 +55,8 @@ PeriodKernel lookup_period_w16(int, bool, bool);
 PeriodKernel lookup_period_w3(int, bool, bool);
 PeriodKernel lookup_period_w6(int, bool, bool);
 PeriodKernel lookup_period_w12(int, bool, bool);
+PeriodKernel lookup_period_w32(int, bool, bool);
+PeriodKernel lookup_period_w64(int, bool, bool);
 
 PeriodKernel lookup_period(int W, int gm, bool bf16, bool post) {
   switch (W) {
@@ -62,6 +68,8 @@ PeriodKernel lookup_period(int W, int gm, bool bf16, bool post) {
     case 3: return lookup_period_w3(gm, bf16, post);
     case 6: return lookup_period_w6(gm, bf16, post);
     case 12: return lookup_period_w12(gm, bf16, post);
+    case 32: return lookup_period_w32(gm, bf16, post);
+    case 64: return lookup_period_w64(gm, bf16, post);
     default: return lookup_period_w0(gm, bf16, post);
   }
 }

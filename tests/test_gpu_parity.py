@@ -665,10 +665,11 @@ def test_streamed_run_equals_upload_run_download(W, n, H, T, grad, fusion, chunk
 
 @pytest.mark.parametrize("W", [32, 48, 64])
 def test_worker_counts_of_whole_tiles(W):
-    """W = 32, 48, 64 (run-time worker counts made of whole tiles of 16 replicas, summed by the
-    constant-index tree and pushed into the run-time counter as aligned blocks): the result is the
-    adjacent-pair tree over all W workers, bitwise, for the stand-alone synchronisation, both
-    fusions, supplied gradient tables and manual call sequences."""
+    """Large worker counts — 32 and 64 with their own instantiation, 48 through the run-time path,
+    where whole tiles of 16 replicas are summed by the constant-index tree and pushed into the
+    run-time counter as aligned blocks: the result is the adjacent-pair tree over all W workers,
+    bitwise, for the stand-alone synchronisation, both fusions, supplied gradient tables and
+    manual call sequences."""
     import torch
     n, H = 1537, 3
     arr = _arrays(n, W)
