@@ -487,14 +487,15 @@ def test_random_call_sequences_match_oracle(seed):
     state round trips and rule changes at period boundaries, mirrored on the oracle."""
     rng = np.random.default_rng(seed)
     n = int(rng.integers(1, 5000))
-    W = int(rng.choice([1, 2, 3, 4, 8, 16, 6]))
+    W = int(rng.choice([1, 2, 3, 4, 8, 16, 6, 5, 12, 32]))
     H = int(rng.integers(1, 7))
     arr = _arrays(n, seed)
     grad = ["noise", "noise_scaled", "quadratic"][seed % 3]
     g, o = make_pair(n, W, 0.05, 0.7, H, grad, seed=seed, arrays=arr, sigma=0.4, b0sq=0.5)
     rule = 0
+    import torch
     for _ in range(40):
-        op = rng.integers(0, 8)
+        op = rng.integers(0, 9)
         if op <= 2:
             T = int(rng.integers(0, 3 * H + 2))
             g.run(T); o.run(T)
@@ -514,6 +515,16 @@ def test_random_call_sequences_match_oracle(seed):
             i = int(rng.integers(0, W))
             x, b2, bs = g.read_state(i)
             g.write_state(i, x, b2, bs)                          # a checkpoint round trip changes nothing
+        elif op == 8:                                            # a complete iteration with a supplied gradient table
+            bf16 = bool(rng.integers(0, 2))
+            G = torch.from_numpy(rng.standard_normal((W, n)).astype(np.float32))
+            G = G.to(torch.bfloat16) if bf16 else G
+            Gd = G.cuda()
+            g.step_grads(Gd.data_ptr(), la.LA_BF16 if bf16 else la.LA_F32)
+            o.local_step(G.float().numpy())
+            if rule != 2 and o.counters()[1] == H:
+                o.sync()
+            g.sync_stream()
         assert g.get_counters() == o.counters()
     compare(g, o, W, TOL_RUN)
 
