@@ -91,3 +91,15 @@ def test_arena_bytes(lib):
     # stride = N rounded up to 64 floats; (2W + 4) arrays of stride floats
     assert la.LocalAdaAlter.arena_bytes([100], 4) == 128 * (2 * 4 + 4) * 4
     assert la.LocalAdaAlter.arena_bytes([64, 64], 1) == 128 * 6 * 4
+
+
+def test_ncu_figures_in_bench_belong_to_the_current_kernel_sources():
+    """bench.py reports ncu-derived figures (DRAM traffic per launch, lane-instructions per update)
+    only while the kernel sources hash to the version they were captured on; this keeps the hash and
+    the sources together: after a kernel change, re-capture (profiles/) and update the constants."""
+    import bench
+    assert bench.kernel_source_hash() == bench.KERNEL_HASH_AT_CAPTURE
+    for name in os.listdir(os.path.join(ROOT, "profiles")):
+        if name.startswith("la_") and name.endswith(".md"):
+            with open(os.path.join(ROOT, "profiles", name)) as f:
+                assert bench.KERNEL_HASH_AT_CAPTURE in f.read(), name
