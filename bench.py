@@ -44,7 +44,7 @@ NOMINAL_HBM_GBS = 8000.0
 #                                 much to save and restore around ncu's replay passes) and scaled by
 #                                 400 007 886 / 2^25 — every byte is touched once, so traffic grows with N.
 #   PERIOD_LANE_INSTR_PER_UPDATE  smsp__inst_executed.sum x 32 / updates per la_period launch
-KERNEL_HASH_AT_CAPTURE = "c624b8026b211464"
+KERNEL_HASH_AT_CAPTURE = "b34d9d2b3173b51e"
 NCU_TRAFFIC_BYTES = {"c2": 2.2235e9, "c5": 29.742e9}
 PERIOD_LANE_INSTR_PER_UPDATE = {"c2": 43.15, "c5": 50.89}   # c5: captured at N = 2^25 (the count per update does not depend on N)
 
@@ -733,8 +733,8 @@ def run_report(args):
 
 def run_kernel_report(args):
     """Per-kernel GB/s away from the benchmark configurations: worker counts with their own
-    instantiation (3, 6, 12), worker counts known only at run time (5, 24, 32, 64), and
-    caller-supplied gradient tables in fp32 and bf16 (W = 4, 8, 16).  N = 2^24 (more for W < 4), pure-noise gradients
+    instantiation (1 ... 16, 32, 64), worker counts known only at run time (17, 20, 24, 48), and
+    caller-supplied gradient tables in fp32 and bf16 (W = 2, 4, 8, 16).  N = 2^24 (more for W < 4), pure-noise gradients
     (the shape of configuration 4), every pass timed by CUDA events around the launch.
     Markdown table to stdout, JSON to --report-out."""
     import torch
@@ -890,8 +890,8 @@ def main():
     ap.add_argument("--tradeoff", action="store_true", help="quality/time against H on a noisy quadratic (table)")
     ap.add_argument("--report-kernels", action="store_true",
                     help="per-kernel GB/s for worker counts and gradient tables outside the five configurations")
-    ap.add_argument("--workers", type=lambda v: [int(x) for x in v.split(",")], default=[3, 6, 12, 5, 24, 32, 64, 4, 8, 16])
-    ap.add_argument("--table-workers", type=lambda v: [int(x) for x in v.split(",")], default=[4, 8, 16])
+    ap.add_argument("--workers", type=lambda v: [int(x) for x in v.split(",")], default=[1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, 16, 32, 64, 17, 20, 24, 48])
+    ap.add_argument("--table-workers", type=lambda v: [int(x) for x in v.split(",")], default=[2, 4, 8, 16])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 

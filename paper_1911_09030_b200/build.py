@@ -21,7 +21,8 @@ OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "liblocal_adaalter.so")
 NVCC = os.environ.get("NVCC", "nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-         "-fmad=false", "-Xcompiler", "-fPIC", "-Xcompiler", "-O2"]
+         "-fmad=false", "-Xcompiler", "-fPIC", "-Xcompiler", "-O2",
+         "-Xfatbin=-compress-all"]   # every worker count up to 16 has its own kernels: keep the image small
 
 
 def _sources():
@@ -46,6 +47,9 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
     FLAGS = globals()["FLAGS"] + (["-DLA_DEBUG"] if debug else [])
     os.makedirs(OBJ, exist_ok=True)
     srcs, deps = _sources(), _deps()
+    if debug:  # the checked build instantiates the first set of worker counts only (compile time)
+        keep = {"la_sweep_w%d.cu" % w for w in (0, 1, 2, 3, 4, 6, 8, 12, 16)}
+        srcs = [s for s in srcs if not os.path.basename(s).startswith("la_sweep_w") or os.path.basename(s) in keep]
     jobs = []
     for s in srcs:
         o = os.path.join(OBJ, os.path.basename(s)[:-3] + ".o")

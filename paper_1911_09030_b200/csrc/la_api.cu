@@ -29,6 +29,14 @@ SweepKernel lookup_sweep_w6(int, int, bool, bool, bool, bool, int);
 SweepKernel lookup_sweep_w12(int, int, bool, bool, bool, bool, int);
 SweepKernel lookup_sweep_w32(int, int, bool, bool, bool, bool, int);
 SweepKernel lookup_sweep_w64(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w5(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w7(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w9(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w10(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w11(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w13(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w14(int, int, bool, bool, bool, bool, int);
+SweepKernel lookup_sweep_w15(int, int, bool, bool, bool, bool, int);
 
 SweepKernel lookup_sweep(int W, int rule, int gm, bool bf16, bool pre, bool step, bool post, int xch) {
   switch (W) {
@@ -40,9 +48,30 @@ SweepKernel lookup_sweep(int W, int rule, int gm, bool bf16, bool pre, bool step
     case 3: return lookup_sweep_w3(rule, gm, bf16, pre, step, post, xch);
     case 6: return lookup_sweep_w6(rule, gm, bf16, pre, step, post, xch);
     case 12: return lookup_sweep_w12(rule, gm, bf16, pre, step, post, xch);
+#ifndef LA_DEBUG   // the checked build keeps to the first set of instantiations; the rest runs as a run-time count
     case 32: return lookup_sweep_w32(rule, gm, bf16, pre, step, post, xch);
     case 64: return lookup_sweep_w64(rule, gm, bf16, pre, step, post, xch);
+    case 5: return lookup_sweep_w5(rule, gm, bf16, pre, step, post, xch);
+    case 7: return lookup_sweep_w7(rule, gm, bf16, pre, step, post, xch);
+    case 9: return lookup_sweep_w9(rule, gm, bf16, pre, step, post, xch);
+    case 10: return lookup_sweep_w10(rule, gm, bf16, pre, step, post, xch);
+    case 11: return lookup_sweep_w11(rule, gm, bf16, pre, step, post, xch);
+    case 13: return lookup_sweep_w13(rule, gm, bf16, pre, step, post, xch);
+    case 14: return lookup_sweep_w14(rule, gm, bf16, pre, step, post, xch);
+    case 15: return lookup_sweep_w15(rule, gm, bf16, pre, step, post, xch);
+#endif
     default: return lookup_sweep_w0(rule, gm, bf16, pre, step, post, xch);
+  }
+}
+
+// True for worker counts without an instantiation of their own.
+bool lookup_sweep_is_runtime(int W) {
+  switch (W) {
+    case 1: case 2: case 3: case 4: case 6: case 8: case 12: case 16: return false;
+#ifndef LA_DEBUG
+    case 5: case 7: case 9: case 10: case 11: case 13: case 14: case 15: case 32: case 64: return false;
+#endif
+    default: return true;
   }
 }
 
@@ -57,6 +86,14 @@ PeriodKernel lookup_period_w6(int, bool, bool);
 PeriodKernel lookup_period_w12(int, bool, bool);
 PeriodKernel lookup_period_w32(int, bool, bool);
 PeriodKernel lookup_period_w64(int, bool, bool);
+PeriodKernel lookup_period_w5(int, bool, bool);
+PeriodKernel lookup_period_w7(int, bool, bool);
+PeriodKernel lookup_period_w9(int, bool, bool);
+PeriodKernel lookup_period_w10(int, bool, bool);
+PeriodKernel lookup_period_w11(int, bool, bool);
+PeriodKernel lookup_period_w13(int, bool, bool);
+PeriodKernel lookup_period_w14(int, bool, bool);
+PeriodKernel lookup_period_w15(int, bool, bool);
 
 PeriodKernel lookup_period(int W, int gm, bool bf16, bool post) {
   switch (W) {
@@ -68,8 +105,18 @@ PeriodKernel lookup_period(int W, int gm, bool bf16, bool post) {
     case 3: return lookup_period_w3(gm, bf16, post);
     case 6: return lookup_period_w6(gm, bf16, post);
     case 12: return lookup_period_w12(gm, bf16, post);
+#ifndef LA_DEBUG   // the checked build keeps to the first set of instantiations; the rest runs as a run-time count
     case 32: return lookup_period_w32(gm, bf16, post);
     case 64: return lookup_period_w64(gm, bf16, post);
+    case 5: return lookup_period_w5(gm, bf16, post);
+    case 7: return lookup_period_w7(gm, bf16, post);
+    case 9: return lookup_period_w9(gm, bf16, post);
+    case 10: return lookup_period_w10(gm, bf16, post);
+    case 11: return lookup_period_w11(gm, bf16, post);
+    case 13: return lookup_period_w13(gm, bf16, post);
+    case 14: return lookup_period_w14(gm, bf16, post);
+    case 15: return lookup_period_w15(gm, bf16, post);
+#endif
     default: return lookup_period_w0(gm, bf16, post);
   }
 }
@@ -453,7 +500,11 @@ int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t
   // threads.  The pure averaging kernel runs best with one group per thread.
   int step_bps = 16 * (int)c->W * 2 / k.vec;
   step_bps = step_bps < 8 ? 8 : (step_bps > 96 ? 96 : step_bps);
-  const int bps = c->blocks_per_sm > 0 ? c->blocks_per_sm : (step ? step_bps : 4096);
+  // (run-time worker counts: their averaging pass overlaps a group's tail with the next group's
+  // first loads, so it wants a grid-stride grid too — W = 5 / 9 / 20: 0.72 / 0.83 / 0.98 of the copy
+  // bandwidth at 32 blocks per SM against 0.58 / 0.65 / 0.86 with one group per thread)
+  const bool runtime_w = la::lookup_sweep_is_runtime((int)c->W);
+  const int bps = c->blocks_per_sm > 0 ? c->blocks_per_sm : (step ? step_bps : (runtime_w ? 32 : 4096));
   const uint64_t cap = (uint64_t)c->num_sms * (uint64_t)bps;
   if (blocks > cap) blocks = cap;
   int cls = !step ? kClassSync : (post ? kClassStepSync : (pre ? kClassSyncStep : kClassLocal));

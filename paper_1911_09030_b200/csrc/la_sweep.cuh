@@ -432,7 +432,7 @@ template <int GM, int V, int CH>
 __device__ __forceinline__ void load_grads(GradChunk<V, CH>& gc, const SweepParams& p, uint64_t& g_addr,
                                            uint64_t row_bytes, uint32_t W, uint32_t i0, uint64_t off) {
   constexpr bool kF32 = (GM == kGradExternalF32);
-  constexpr uint32_t kElem = kF32 ? 4u : 2u;
+  [[maybe_unused]] constexpr uint32_t kElem = kF32 ? 4u : 2u;
 #pragma unroll
   for (int k = 0; k < CH; ++k)
     if (i0 + k < W) {
@@ -600,14 +600,20 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
   const uint64_t g_base = reinterpret_cast<uint64_t>(p.gext);
   const uint64_t g_row_bytes = p.n * kGradElem;
 
-  ReplicaChunk<V, CH> nxt;
-  GradChunk<V, kExternal ? CH : 1> gnxt;
+  // Static worker counts: one buffer of loads in flight (`nxt`), copied when consumed — the chunk
+  // loop is fully unrolled, so the copies are register renaming.  Run-time worker counts: the loop
+  // stays rolled, a copy would wait for the data BEFORE the next loads are issued, so there are
+  // two buffers with compile-time roles (`rb[0]`, `rb[1]`: slots of even and odd position).
+  ReplicaChunk<V, CH> nxt, rb[(WR_ > 0) ? 1 : 2];
+  GradChunk<V, kExternal ? CH : 1> gnxt, gb[(WR_ > 0) ? 1 : 2];
   CoordInputs<V> in_next;
   load_coord<GM, STEP, kLoadsBs, V>(in_next, p, grp * V);
   uint64_t ld_addr = rd_base + grp * (V * sizeof(float));
   uint64_t g_addr = g_base + grp * (V * kGradElem);
-  load_chunk<V, CH, ACC>(nxt, ld_addr, rd_b_delta, stride_bytes, Wr, 0u LA_DBG_ARG(rd_base + grp * (V * sizeof(float))));
-  if (kExternal) load_grads<GM, V, kExternal ? CH : 1>(gnxt, p, g_addr, g_row_bytes, W, 0u, grp * V);
+  load_chunk<V, CH, ACC>((WR_ > 0) ? nxt : rb[0], ld_addr, rd_b_delta, stride_bytes, Wr, 0u
+                         LA_DBG_ARG(rd_base + grp * (V * sizeof(float))));
+  if (kExternal)
+    load_grads<GM, V, kExternal ? CH : 1>((WR_ > 0) ? gnxt : gb[0], p, g_addr, g_row_bytes, W, 0u, grp * V);
 
   // A step that follows an average takes supplied gradients in its write loop, kWriteChunk table rows ahead.
   constexpr bool kSuppliedAfterAverage = kSupplied && PRE;
@@ -673,33 +679,85 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
 #pragma unroll kReadUnroll
       for (uint32_t i0 = 0; i0 < Wr; i0 += CH) chunk(i0, tree, i0, i0 + CH <= Wr);
     } else {
-      // Worker count known only at run time.  Passes that average first take whole tiles of
-      // kTile replicas: inside a tile every position is a compile-time constant, so the tile is
-      // summed by the stack-form tree (constant register indices, no predication) and enters the
-      // run-time counter as one aligned block — an aligned block of 2^k workers is a complete
-      // subtree of the adjacent-pair tree.  What is left (fewer than kTile replicas) goes through
-      // the counter chunk by chunk.
+      // Worker count known only at run time.  The replicas are consumed in SLOTS of CH, always an
+      // even number of them per coordinate group, so that every slot has a compile-time position
+      // (even: buffer 0, odd: buffer 1): a slot first starts the loads of the slot that follows
+      // into the other buffer, then consumes its own.  Only the last (odd) slot of a group has
+      // nothing after it in the group; it fetches the first chunk of the thread's next group.
+      auto slot = [&](auto position, const uint32_t i0, auto& tr, const uint32_t local0, const bool whole)
+                      __attribute__((always_inline)) {
+        constexpr int P = decltype(position)::value;
+        ReplicaChunk<V, CH>& cur = rb[P];
+        ReplicaChunk<V, CH>& ahead = rb[1 - P];
+        GradChunk<V, kExternal ? CH : 1>& gcur = gb[P];
+        GradChunk<V, kExternal ? CH : 1>& gahead = gb[1 - P];
+        if (i0 + CH < Wr) {
+          load_chunk<V, CH, ACC>(ahead, ld_addr, rd_b_delta, stride_bytes, Wr, i0 + CH LA_DBG_ARG(rd_base + off * sizeof(float)));
+          if (kExternal) load_grads<GM, V, kExternal ? CH : 1>(gahead, p, g_addr, g_row_bytes, W, i0 + CH, off);
+        } else if (P == 1 && has_next) {
+          load_coord<GM, STEP, kLoadsBs, V>(in_next, p, next_grp * V);
+          ld_addr = rd_base + next_grp * (V * sizeof(float));
+          load_chunk<V, CH, ACC>(ahead, ld_addr, rd_b_delta, stride_bytes, Wr, 0u LA_DBG_ARG(rd_base + next_grp * (V * sizeof(float))));
+          if (kExternal) {
+            g_addr = g_base + next_grp * (V * kGradElem);
+            load_grads<GM, V, kExternal ? CH : 1>(gahead, p, g_addr, g_row_bytes, W, 0u, next_grp * V);
+          }
+        }
+        asm volatile("" ::: "memory");
+#pragma unroll
+        for (int k = 0; k < CH; ++k)
+          if (whole || i0 + k < Wr) {
+            const uint32_t i = i0 + k;
+            if (PRE) {
+              tr.push_in_chunk(local0 + k, k, whole, cur.x[k], cur.b[k]);
+            } else {
+              const Vec<V> g = kExternal ? gcur.g[kExternal ? k : 0]
+                                         : gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
+              apply<V, ACC>(r, g, cur.x[k], cur.b[k]);
+              if (POST) {
+                tr.push_in_chunk(local0 + k, k, whole, cur.x[k], cur.b[k]);
+              } else {
+                store_replica<V, ACC>(st_addr, b_delta, stride_bytes, cur.x[k], cur.b[k]
+                                      LA_DBG_ARG(x_base + off * sizeof(float) + (uint64_t)i * stride_bytes));
+              }
+            }
+          }
+      };
+      using Even = std::integral_constant<int, 0>;
+      using Odd = std::integral_constant<int, 1>;
+      // Passes that average first take whole tiles of kTile replicas: inside a tile every position
+      // is a compile-time constant, so the tile is summed by the stack-form tree (constant register
+      // indices, no predication) and enters the run-time counter as one aligned block — an aligned
+      // block of 2^k workers is a complete subtree of the adjacent-pair tree.  What is left (fewer
+      // than half a tile) goes through the counter in one last pair of slots.
       constexpr int kTile = 16, kTileLog = 4;
-      static_assert(kTile % CH == 0 && (kTile / 2) % CH == 0, "tiles are whole chunks");
+      static_assert(CH == 4, "tiles and half tiles are whole pairs of slots");
       uint32_t i0 = 0;
       if ((PRE || POST) && V == 2) {  // (four-coordinate threads have no registers to spare for a tile)
         for (; i0 + kTile <= Wr; i0 += kTile) {
           PairTree<V, ACC> tile;
-#pragma unroll
-          for (int c = 0; c < kTile / CH; ++c) chunk(i0 + c * CH, tile, c * CH, true);
+          slot(Even{}, i0, tile, 0u, true);
+          slot(Odd{}, i0 + CH, tile, (uint32_t)CH, true);
+          slot(Even{}, i0 + 2 * CH, tile, (uint32_t)(2 * CH), true);
+          slot(Odd{}, i0 + 3 * CH, tile, (uint32_t)(3 * CH), true);
           tile.finish(kTile);
           tree.template push_block<kTileLog>(tile.x[0], tile.b[0]);
         }
         if (i0 + kTile / 2 <= Wr) {  // one half tile, the same way
           PairTree<V, ACC> tile;
-#pragma unroll
-          for (int c = 0; c < kTile / 2 / CH; ++c) chunk(i0 + c * CH, tile, c * CH, true);
+          slot(Even{}, i0, tile, 0u, true);
+          slot(Odd{}, i0 + CH, tile, (uint32_t)CH, true);
           tile.finish(kTile / 2);
           tree.template push_block<kTileLog - 1>(tile.x[0], tile.b[0]);
           i0 += kTile / 2;
         }
       }
-      for (; i0 < Wr; i0 += CH) chunk(i0, tree, i0, i0 + CH <= Wr);
+      // (a group that ended exactly on a tile has had its last odd slot; otherwise pairs of slots
+      // until the replicas are used up — the odd slot of the last pair may be empty)
+      for (; i0 < Wr; i0 += 2 * CH) {
+        slot(Even{}, i0, tree, i0, i0 + CH <= Wr);
+        slot(Odd{}, i0 + CH, tree, i0 + CH, i0 + 2 * CH <= Wr);
+      }
     }
 
     if (PRE || POST) {

@@ -55,7 +55,7 @@ def test_tails_and_worker_counts(n, W):
         g.close()
 
 
-@pytest.mark.parametrize("W", [5, 6, 7, 11, 13, 24, 32, 40, 48, 64])
+@pytest.mark.parametrize("W", [5, 6, 7, 9, 10, 11, 13, 14, 15, 17, 20, 23, 24, 29, 32, 40, 48, 63, 64])
 def test_generic_worker_counts(W):
     n, T = 257, 9
     arr = _arrays(n, W)
@@ -487,7 +487,7 @@ def test_random_call_sequences_match_oracle(seed):
     state round trips and rule changes at period boundaries, mirrored on the oracle."""
     rng = np.random.default_rng(seed)
     n = int(rng.integers(1, 5000))
-    W = int(rng.choice([1, 2, 3, 4, 8, 16, 6, 5, 12, 32]))
+    W = int(rng.choice([1, 2, 3, 4, 8, 16, 6, 5, 12, 32, 17, 20]))
     H = int(rng.integers(1, 7))
     arr = _arrays(n, seed)
     grad = ["noise", "noise_scaled", "quadratic"][seed % 3]
