@@ -289,6 +289,10 @@ int la_comm_import(la_ctx* ctx);
 int la_comm_step_export(la_ctx* ctx);
 int la_comm_step_grads_export(la_ctx* ctx, const void* g_dev, int dtype);
 int la_comm_import_step(la_ctx* ctx);
+/* la_comm_import_step with caller-supplied gradients for the step t' = 1 (table as for
+ * la_local_step_grads): together with la_comm_step_grads_export a trainer's synchronisation
+ * costs no pass over the replicas of its own. */
+int la_comm_import_step_grads(la_ctx* ctx, const void* g_dev, int dtype);
 /* Verification aid for the synthetic gradient source (not part of the paper's method): the two
  * building blocks of the normal draw, exactly as the sweep kernels evaluate them, over their whole
  * 24-bit domains, so that they can be compared element by element with another implementation:

@@ -1435,6 +1435,21 @@ int la_comm_import_step(la_ctx* c) {
   return LA_OK;
 }
 
+int la_comm_import_step_grads(la_ctx* c, const void* g_dev, int dtype) {
+  if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
+  if (!c->S) return fail(c, LA_ESTATE, "call la_comm_create first");
+  if (!g_dev) return fail(c, LA_EINVAL, "g_dev is NULL");
+  if (dtype != LA_F32 && dtype != LA_BF16) return fail(c, LA_EINVAL, "dtype must be LA_F32 or LA_BF16");
+  if (c->rule != LA_RULE_ADAALTER) return fail(c, LA_ESTATE, "sharding by worker is implemented for Local AdaAlter only");
+  DeviceGuard guard(c->device);
+  { int rc_ = import_pending_sums(c); if (rc_) return rc_; }
+  int rc = launch_sweep(c, true, true, false, c->t + 1, 1u, dtype == LA_F32 ? la::kGradExternalF32 : la::kGradExternalBF16,
+                        g_dev, 2);
+  if (rc) return rc;
+  c->nsync += 1; c->t += 1; c->tp = 1;
+  return LA_OK;
+}
+
 int la_diagnostics(la_ctx* c, double* objective, double* replica_spread) {
   if (!c) return fail(nullptr, LA_EINVAL, "ctx is NULL");
   DeviceGuard guard(c->device);

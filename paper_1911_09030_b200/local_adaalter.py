@@ -105,6 +105,7 @@ def lib() -> C.CDLL:
             "la_comm_step_export": [vp],
             "la_comm_step_grads_export": [vp, vp, i32],
             "la_comm_import_step": [vp],
+            "la_comm_import_step_grads": [vp, vp, i32],
             "la_stream_sync": [vp],
             "la_noise_tables": [vp, vp, vp, vp],
             "la_replica_means_static": [vp, vp, u32, u64, u64, vp, vp, vp],
@@ -416,3 +417,6 @@ class LocalAdaAlter:
 
     def comm_import_step(self):
         self._ck(self.L.la_comm_import_step(self.h))
+
+    def comm_import_step_grads(self, g_dev_ptr, dtype=LA_F32):
+        self._ck(self.L.la_comm_import_step_grads(self.h, C.c_void_p(int(g_dev_ptr)), int(dtype)))

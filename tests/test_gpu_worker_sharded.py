@@ -286,9 +286,18 @@ def test_fused_exchange_steps_with_emulated_ranks(world, W_local, grad):
             t += 1
             if closes:
                 exchange()
-                for g in ctxs:
-                    g.comm_import()
                 o.sync()
+                if t < T:                         # the next iteration starts from the exchanged totals, in one pass
+                    G = rng.standard_normal((W_total, n)).astype(np.float32)
+                    o.local_step(G)
+                    for r, g in enumerate(ctxs):
+                        Gd = torch.from_numpy(G[r * W_local:(r + 1) * W_local].copy()).cuda()
+                        g.comm_import_step_grads(Gd.data_ptr(), la.LA_F32)
+                        g.stream_sync()
+                    t += 1
+                else:
+                    for g in ctxs:
+                        g.comm_import()
             continue
         if closes:
             for g in ctxs:
