@@ -44,7 +44,7 @@ NOMINAL_HBM_GBS = 8000.0
 #                                 much to save and restore around ncu's replay passes) and scaled by
 #                                 400 007 886 / 2^25 — every byte is touched once, so traffic grows with N.
 #   PERIOD_LANE_INSTR_PER_UPDATE  smsp__inst_executed.sum x 32 / updates per la_period launch
-KERNEL_HASH_AT_CAPTURE = "b34d9d2b3173b51e"
+KERNEL_HASH_AT_CAPTURE = "692c9f8935aee566"
 NCU_TRAFFIC_BYTES = {"c2": 2.2235e9, "c5": 29.742e9}
 PERIOD_LANE_INSTR_PER_UPDATE = {"c2": 43.15, "c5": 50.89}   # c5: captured at N = 2^25 (the count per update does not depend on N)
 
@@ -873,6 +873,7 @@ def main():
     ap.add_argument("--workload", default="c5", help="c1..c5; default: the largest single-GPU configuration")
     ap.add_argument("--H", type=int, default=None, help="override the synchronisation period")
     ap.add_argument("--T", type=int, default=None, help="override iterations per step")
+    ap.add_argument("--W", type=int, default=None, help="override the worker count (replicas per rank)")
     ap.add_argument("--N", type=int, default=None, help="override the size (one flat tensor), e.g. for small ncu captures")
     ap.add_argument("--fusion", type=int, default=4,
                     help="0 unfused, 1 step+sync, 2 sync+next step, 3 temporal blocking, 4 synchronised state stored once")
@@ -909,6 +910,8 @@ def main():
         wl.T = args.T
     if args.N is not None:
         wl.sizes = [args.N]
+    if args.W is not None:
+        wl.W = args.W
     if args.impl == "reference":
         run_reference(args, wl)
     elif args.sharding == "worker":

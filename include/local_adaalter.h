@@ -147,7 +147,7 @@ int la_set_rule(la_ctx* ctx, int rule);
 int la_set_fusion(la_ctx* ctx, int mode);
 /* Tuning knob: the sweep kernels run as a grid-stride loop over at most
  * blocks_per_sm * (number of SMs) blocks of 256 threads; 0 restores the built-in
- * per-kernel defaults (16 per replica up to 96 for kernels that take a step, 768 for the
+ * per-kernel defaults (16 per replica, between 32 and 96, for kernels that take a step, 768 for the
  * temporal-blocking kernel, unbounded for the pure sync). */
 int la_set_launch_shape(la_ctx* ctx, int blocks_per_sm);
 /* Launch-bound regime (small N, e.g. a 2 MB state where a step takes a few microseconds): let

@@ -497,9 +497,9 @@ int launch_sweep(la_ctx* c, bool pre, bool step, bool post, uint64_t t, uint32_t
   // pays off) yet stays small enough to balance the SMs.  The work of a block grows with the
   // replicas and coordinates a thread owns, so the grid does too: 16 W blocks per SM for
   // two-coordinate threads (W = 4: 64; 96 from W = 6 on), half of that for four-coordinate
-  // threads.  The pure averaging kernel runs best with one group per thread.
+  // threads, never fewer than 32.  The pure averaging kernel runs best with one group per thread.
   int step_bps = 16 * (int)c->W * 2 / k.vec;
-  step_bps = step_bps < 8 ? 8 : (step_bps > 96 ? 96 : step_bps);
+  step_bps = step_bps < 32 ? 32 : (step_bps > 96 ? 96 : step_bps);
   // (run-time worker counts: their averaging pass overlaps a group's tail with the next group's
   // first loads, so it wants a grid-stride grid too — W = 5 / 9 / 20: 0.72 / 0.83 / 0.98 of the copy
   // bandwidth at 32 blocks per SM against 0.58 / 0.65 / 0.86 with one group per thread)
