@@ -68,7 +68,9 @@ enum { LA_RULE_ADAALTER = 0,  /* Algorithm 3, Local AdaAlter (default) */
        LA_RULE_LOCAL_SGD = 1, /* Algorithm 2: y = x - eta G, x averaged every H steps, no accumulator */
        LA_RULE_ADAGRAD = 2 }; /* Algorithm 1: gradients averaged every step, B^2 += G o G, updated B^2 divides */
 #define LA_H_NEVER 0xFFFFFFFFu                  /* H = +infinity: never synchronise */
-#define LA_MAX_WORKERS 64u
+#define LA_MAX_WORKERS 64u                      /* every W up to 16, and 32 and 64, has kernels of its own;
+                                                   other counts run kernels that take W at run time
+                                                   (same results, the passes that average 10-25 % slower) */
 
 /* Extended creation parameters.  Zero-initialise, then fill. */
 typedef struct la_config {
