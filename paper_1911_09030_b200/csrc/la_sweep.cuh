@@ -135,9 +135,9 @@ constexpr int kTreeDepth = 7;  // log2(kMaxWorkers) + 1 partial sums
 #define LA_CH_V4_STEP (LA_CH_V4 < 2 ? 2 : LA_CH_V4)  // from being issued early (bf16 table, W = 4 / 8: 0.94 / 0.95 against 0.89)
 #endif
 #ifndef LA_WRITE_CH_V4
-#define LA_WRITE_CH_V4 1  // table rows fetched ahead by a four-coordinate step that follows an average
-                          // (measured at W = 4 / 8: 1 row 0.83 / 0.76 of the copy bandwidth, 2 rows 0.75 / 0.77,
-                          // 4 rows 0.74 / 0.79; two-coordinate threads with 4-byte table loads 0.55 / 0.62)
+#define LA_WRITE_CH_V4 2  // table rows fetched ahead by a four-coordinate step that follows an average
+                          // (bf16 table, one-copy step at W = 4 / 8 / 16: 1 row 0.92 / 0.94 / 0.95 of the copy
+                          // bandwidth, 2 rows 0.94 / 0.95 / 0.95, 4 rows the same)
 #endif
 constexpr int kBlockThreads = LA_BLOCK;
 
@@ -425,8 +425,24 @@ __device__ __forceinline__ void store_replica(uint64_t& addr, uint64_t b_delta, 
 // while the previous chunk is consumed.
 template <int V, int CH>
 struct GradChunk {
-  Vec<V> g[CH];
+  Vec<V> g[CH];  // fp32 table: the values; bf16 table: the V/2 loaded words in slots 0 .. V/2-1, widened on use
 };
+
+// The gradient values of one row of a chunk.  A bf16 row stays in the packed form it was loaded in
+// until it is used, so that no instruction between a load and its use waits for the data (and a
+// chunk fetched ahead costs half the registers); widening bf16 -> fp32 is exact.
+template <int GM, int V>
+__device__ __forceinline__ Vec<V> unpack_grads(const Vec<V>& raw) {
+  if (GM != kGradExternalBF16) return raw;
+  Vec<V> g;
+#pragma unroll
+  for (int k = 0; k < V; k += 2) {
+    const uint32_t w = __float_as_uint(raw.v[k / 2]);
+    g.v[k] = __uint_as_float(w << 16);
+    g.v[k + 1] = __uint_as_float(w & 0xFFFF0000u);
+  }
+  return g;
+}
 
 template <int GM, int V, int CH>
 __device__ __forceinline__ void load_grads(GradChunk<V, CH>& gc, const SweepParams& p, uint64_t& g_addr,
@@ -448,35 +464,30 @@ __device__ __forceinline__ void load_grads(GradChunk<V, CH>& gc, const SweepPara
         if (kF32) {
           gc.g[k] = ld_stream<V>(as_ptr(g_addr));
         } else {
-          // V bf16 values in one 32- or 64-bit load; widening bf16 -> fp32 is exact
+          // V bf16 values in one 32- or 64-bit load, kept packed (see unpack_grads)
+          gc.g[k] = splat<V>(0.0f);
           if (V == 2) {
-            const uint32_t w = __ldcs(reinterpret_cast<const uint32_t*>(g_addr));
-            gc.g[k].v[0] = __uint_as_float(w << 16);
-            gc.g[k].v[1] = __uint_as_float(w & 0xFFFF0000u);
+            gc.g[k].v[0] = __uint_as_float(__ldcs(reinterpret_cast<const uint32_t*>(g_addr)));
           } else {
             const uint2 w = __ldcs(reinterpret_cast<const uint2*>(g_addr));
-            gc.g[k].v[0] = __uint_as_float(w.x << 16);
-            gc.g[k].v[1] = __uint_as_float(w.x & 0xFFFF0000u);
-            gc.g[k].v[V - 2] = __uint_as_float(w.y << 16);
-            gc.g[k].v[V - 1] = __uint_as_float(w.y & 0xFFFF0000u);
+            gc.g[k].v[0] = __uint_as_float(w.x);
+            gc.g[k].v[1] = __uint_as_float(w.y);
           }
         }
       } else {
+        if (!kF32) gc.g[k] = splat<V>(0.0f);
 #pragma unroll
         for (int e = 0; e < V; ++e) {
-          float v = 0.0f;
           bool take = off + e < p.n;
 #ifdef LA_DEBUG
           take = take && dbg_access_ok(reinterpret_cast<const void*>(g_addr + e * kElem), kElem);
 #endif
-          if (take) {
-            if (kF32) {
-              v = __ldcs(reinterpret_cast<const float*>(g_addr) + e);
-            } else {
-              v = __uint_as_float((uint32_t)__ldcs(reinterpret_cast<const unsigned short*>(g_addr) + e) << 16);
-            }
+          if (kF32) {
+            gc.g[k].v[e] = take ? __ldcs(reinterpret_cast<const float*>(g_addr) + e) : 0.0f;
+          } else {  // element by element into the packed form
+            const uint32_t h = take ? (uint32_t)__ldcs(reinterpret_cast<const unsigned short*>(g_addr) + e) : 0u;
+            gc.g[k].v[e / 2] = __uint_as_float(__float_as_uint(gc.g[k].v[e / 2]) | (h << (16 * (e & 1))));
           }
-          gc.g[k].v[e] = v;
         }
       }
       advance(g_addr, row_bytes);
@@ -662,7 +673,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
           if (PRE) {
             tr.push_in_chunk(local0 + k, k, whole, cur.x[k], cur.b[k]);
           } else {
-            const Vec<V> g = kExternal ? gcur.g[kExternal ? k : 0]
+            const Vec<V> g = kExternal ? unpack_grads<GM, V>(gcur.g[kExternal ? k : 0])
                                        : gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
             apply<V, ACC>(r, g, cur.x[k], cur.b[k]);
             if (POST) {
@@ -711,7 +722,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
             if (PRE) {
               tr.push_in_chunk(local0 + k, k, whole, cur.x[k], cur.b[k]);
             } else {
-              const Vec<V> g = kExternal ? gcur.g[kExternal ? k : 0]
+              const Vec<V> g = kExternal ? unpack_grads<GM, V>(gcur.g[kExternal ? k : 0])
                                          : gradient<GM, BF16, V>(p, in, cur.x[k], kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
               apply<V, ACC>(r, g, cur.x[k], cur.b[k]);
               if (POST) {
@@ -794,7 +805,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_sweep(const SweepParams p) 
               for (int k = 0; k < kWriteChunk; ++k)
                 if (i0 + k < W) {
                   Vec<V> xv = xm, bv = bm;
-                  apply<V, ACC>(r, gcur.g[k], xv, bv);
+                  apply<V, ACC>(r, unpack_grads<GM, V>(gcur.g[k]), xv, bv);
                   store_replica<V, ACC>(st_addr, b_delta, stride_bytes, xv, bv
                                         LA_DBG_ARG(x_base + off * sizeof(float) + (uint64_t)(i0 + k) * stride_bytes));
                 }
@@ -864,7 +875,7 @@ __global__ void __launch_bounds__(LA_BLOCK, MINB) la_adagrad(const SweepParams p
       if (kExternal) {
         GradChunk<V, 1> gc;
         load_grads<GM, V, 1>(gc, p, g_addr, p.n * kGradElem, W, i, off);
-        g = gc.g[0];
+        g = unpack_grads<GM, V>(gc.g[0]);
       } else {
         g = gradient<GM, false, V>(p, in, x, kNeedsNoise ? keys[i] : 0ull, ctr0, i, off);
       }
