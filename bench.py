@@ -44,7 +44,7 @@ NOMINAL_HBM_GBS = 8000.0
 #                                 much to save and restore around ncu's replay passes) and scaled by
 #                                 400 007 886 / 2^25 — every byte is touched once, so traffic grows with N.
 #   PERIOD_LANE_INSTR_PER_UPDATE  smsp__inst_executed.sum x 32 / updates per la_period launch
-KERNEL_HASH_AT_CAPTURE = "37e3e602858f15f9"
+KERNEL_HASH_AT_CAPTURE = "f309962a307aeecc"
 NCU_TRAFFIC_BYTES = {"c2": 2.2235e9, "c5": 29.742e9}
 PERIOD_LANE_INSTR_PER_UPDATE = {"c2": 43.15, "c5": 50.89}   # c5: captured at N = 2^25 (the count per update does not depend on N)
 
