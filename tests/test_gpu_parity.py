@@ -66,6 +66,21 @@ def test_generic_worker_counts(W):
         compare(g, o, W, TOL_RUN)
 
 
+@pytest.mark.parametrize("grad,bf16", [("noise", False), ("noise_scaled", False), ("noise_scaled", True),
+                                       ("quadratic", True), ("constant", False)])
+@pytest.mark.parametrize("W", [5, 6])
+def test_gradient_kinds_with_their_own_register_budget(W, grad, bf16):
+    """W = 5 and 6 compile each gradient kind with the number of resident blocks that suits it;
+    every kind, every fusion mode, several blocks and a ragged tail."""
+    n, H, T = 70003, 3, 8
+    arr = _arrays(n, W)
+    for fusion in (0, 1, 2, 3, 4):
+        g, o = make_pair(n, W, 0.05, 0.7, H, grad, seed=40 + W, arrays=arr, sigma=0.5, bf16=bf16, fusion=fusion)
+        g.run(T)
+        o.run(T)
+        compare(g, o, W, TOL_RUN)
+
+
 @pytest.mark.parametrize("grad,bf16", [("noise", False), ("noise", True), ("noise_scaled", False),
                                        ("noise_scaled", True), ("quadratic", False), ("quadratic", True),
                                        ("constant", False)])
@@ -254,7 +269,8 @@ def test_supplied_gradients_match_oracle(dtype, n):
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("W,n,H,fusion", [(4, 70002, 3, 1), (8, 4098, 2, 0), (16, 1000, 4, 1), (3, 777, 2, 1),
                                            (2, 12, 1, 1), (5, 4100, 3, 2), (4, 70002, 3, 4), (8, 4098, 2, 4),
-                                           (3, 777, 5, 4), (1, 2052, 2, 4), (33, 260, 3, 4), (2, 12, 1, 4)])
+                                           (3, 777, 5, 4), (1, 2052, 2, 4), (33, 260, 3, 4), (2, 12, 1, 4),
+                                           (5, 4100, 3, 4), (6, 4100, 2, 1), (6, 4102, 3, 4), (6, 777, 2, 0)])
 def test_step_grads_full_iteration(dtype, W, n, H, fusion):
     """la_step_grads = local step + the synchronisation when it is due (fused or not); even n takes
     the vector loads, odd n the scalar ones; a table offset by one element is mis-aligned."""
